@@ -1,0 +1,290 @@
+#!/usr/bin/env python
+"""Benchmark of the HiSpec verification path on B200.
+
+One *step* is one super-round of Algorithm 2 on the Llama-3-8B-shaped early-exit
+model (exits 8/16/32, batch 1, prompt 1024, k = N_d = 5, target verification after
+every 2 intermediate rounds): 2 x [6 draft steps through layers [0,8) + one
+intermediate verification of 6 rows through [8,16)] + one target verification of
+the tentatively accepted rows through [16,32).  Every step of it runs in the
+library's CUDA kernels, called through the C ABI.
+
+  value   verified tokens/s: tokens committed after target verification divided by
+          the device time of K steps, all inputs resident in HBM, no host round trip;
+  e2e     the same metric through the public driver with host buffers: per step the
+          host reads the step's result record (device -> pinned host) and the tokens
+          are assembled on the host; prompt ids are uploaded from pinned host memory
+          (inside the timed region the per-step input is the pending token, which the
+          device already holds, so h2d bytes per step are 0 after the prompt);
+  roofline  projections (the dominant kernel): weight bytes streamed / summed event
+          time of the bracketed launches, against the measured HBM copy bandwidth;
+  cpu_baseline  the fp32 CPU oracle timed on one super-round of the same shape.
+
+`--impl reference` times the oracle alone (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified tokens/s per B200 (HiSpec, Llama-3-8B shape, batch 1, k=5)"
+UNIT = "tokens/s"
+N_PROMPT, N_D, ROUNDS = 1024, 5, 2
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            j = json.load(open(p))
+            return float(j["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.stop_flag = index, [], False
+
+    def run(self):
+        while not self.stop_flag:
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 6:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            time.sleep(0.05)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        sm = sorted(int(float(s[0])) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": int(float(self.samples[0][1])), "reasons": reasons,
+                "samples": len(sm)}
+
+
+def algorithmic_bytes_super_round(shape, ctx_len: int) -> float:
+    """What one super-round must move: weights of each call's layer range + head, KV read/write, hidden rows."""
+    W, H, kvb = shape.layer_weight_bytes, shape.head_bytes, shape.kv_bytes_per_token_layer
+    d4 = shape.d_model * 4
+    draft = shape.L_d * W + H + shape.L_d * kvb * (ctx_len + 1) + d4
+    vi = (shape.L_i - shape.L_d) * W + H + (shape.L_i - shape.L_d) * kvb * (ctx_len + N_D + 1) + 2 * (N_D + 1) * d4
+    rows_t = ROUNDS * (N_D + 1)
+    vt = (shape.L_f - shape.L_i) * W + H + (shape.L_f - shape.L_i) * kvb * (ctx_len + rows_t) + rows_t * d4
+    return ROUNDS * ((N_D + 1) * draft + vi) + vt
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_2510_01336_b200 import binding, workload as wl
+    from paper_2510_01336_b200.driver import HiSpecLoop
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    shape = wl.L3_8B
+    t0 = time.time()
+    w = wl.make_weights(shape, device="cuda")
+    max_rows = ROUNDS * (N_D + 1) + 1
+    n_super = args.warmup + 2 * args.steps + 16
+    max_ctx = N_PROMPT + n_super * ROUNDS * (N_D + 1) + 64
+    max_pages = (max_ctx + 15) // 16
+    ctx = binding.Context(shape, w, page_size=16, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    st = ctx.new_state(1, max_pages, wl.make_block_table(shape, 1, max_pages))
+    loop = HiSpecLoop(ctx, st, 1, N_D, ROUNDS)
+    prompt_host = wl.make_tokens(shape, N_PROMPT).pin_memory()
+    loop.prefill([prompt_host.tolist()])
+    setup_s = time.time() - t0
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(n_steps, host_roundtrip):
+        l0 = int(st.len_target[0])
+        n0 = ctx.launch_count()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        wall0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(n_steps):
+            loop.enqueue_super_round()
+            if host_roundtrip:
+                loop.collect()
+        e1.record(stream)
+        barrier()
+        wall = time.perf_counter() - wall0
+        ms = e0.elapsed_time(e1)
+        if host_roundtrip:
+            ms = max(ms, wall * 1e3)
+        toks = int(st.len_target[0]) - l0
+        return ms, toks, ctx.launch_count() - n0
+
+    for _ in range(max(args.warmup, 3)):
+        loop.enqueue_super_round()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms, toks, launches = timed(args.steps, False)
+    sampler.stop_flag = True
+    ms_e2e, toks_e2e, _ = timed(args.steps, True)
+    status = ctx.status()
+
+    # roofline of the projection kernel: event-bracketed launches over a few more super-rounds
+    ctx.profile_enable(True)
+    for _ in range(min(args.steps, 4)):
+        loop.enqueue_super_round()
+    g_ms, g_bytes, g_n = ctx.profile_read(0)
+    a_ms, _, a_n = ctx.profile_read(1)
+    ctx.profile_enable(False)
+    peak, peak_kind = peaks()
+    achieved = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms, ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        c = torch.tensor([float(toks), float(toks_e2e)], device="cuda")
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        ms, ms_e2e = t.tolist()
+        toks, toks_e2e = c.tolist()
+    if rank != 0:
+        return
+    ctx_len = N_PROMPT + args.warmup * 2
+    step_bytes = algorithmic_bytes_super_round(shape, ctx_len)
+    line = {
+        "metric": METRIC, "value": toks / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "configs[1]: Llama-3-8B-shaped early-exit model, exits 8/16/32, batch 1, prompt 1024 "
+                               "uniform-random tokens, k=5 greedy drafts, target every 2 intermediate rounds; "
+                               "bf16 N(0,0.02) weights (literal: near-zero acceptance)",
+                   "step": "one super-round: 2 x (6 draft steps + verify-I) + verify-T", "replicas": world,
+                   "l2": "inputs larger than L2 (each call streams >= 4.5 GB of weights)",
+                   "activations": "bf16 hi+lo split", "tokens_committed": toks,
+                   "algorithmic_gb_per_step": step_bytes / 1e9,
+                   "step_hbm_gbs": step_bytes / 1e9 / (ms / args.steps * 1e-3), "device_status": status,
+                   "setup_s": round(setup_s, 1)},
+        "clocks": sampler.summary(),
+        "e2e": {"value": toks_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 4 * (2 + max_rows + ROUNDS), "ms_per_step": ms_e2e / args.steps,
+                "prompt_h2d_bytes": 4 * N_PROMPT},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "kernel": "gemm_tc_kernel (all projections + exit head)",
+                     "launches": g_n, "avg_launch_us": 1e3 * g_ms / max(g_n, 1), "peak_source": f"of {peak_kind}",
+                     "attention_ms_share": a_ms / max(a_ms + g_ms, 1e-9)},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        del loop, ctx, st
+        torch.cuda.empty_cache()
+        line["cpu_baseline"] = cpu_super_round(shape, w, budget_steps=1)
+    print(json.dumps(line), flush=True)
+
+
+def cpu_super_round(shape, w_gpu, budget_steps: int):
+    """The oracle, as it stands, timed on one super-round of the same shape from a synthetic cached state
+    (K/V of all layers for 1024 positions drawn N(0,1): a CPU prefill of 1024 tokens would take hours)."""
+    import numpy as np
+    import torch
+    from oracle import hispec as orc
+    from paper_2510_01336_b200 import workload as wl
+
+    w = w_gpu.to("cpu") if w_gpu is not None else wl.make_weights(shape)
+    m = orc.OracleModel.from_weights(w, kv_round_bf16=True)
+    hs = orc.HiSpecOracle(m, shape.L_d, shape.L_i, shape.L_f)
+    rows = ROUNDS * (N_D + 1) + 1
+    st = hs.new_state(N_PROMPT + 4 * rows, rows)
+    rng = np.random.default_rng(shape.seed + 4000)
+    for l in range(shape.n_layers):
+        st.cache.k[l, :N_PROMPT] = rng.standard_normal(st.cache.k[l, :N_PROMPT].shape, dtype=np.float32)
+        st.cache.v[l, :N_PROMPT] = rng.standard_normal(st.cache.v[l, :N_PROMPT].shape, dtype=np.float32)
+    st.len_d = st.len_i = st.len_f = N_PROMPT
+    pending = int(wl.make_tokens(shape, 1, seed_offset=5000)[0])
+    times, committed = [], 0
+    for _ in range(budget_steps):
+        t0 = time.perf_counter()
+        V = []
+        for _r in range(ROUNDS):
+            S, u = [], pending
+            for j in range(N_D + 1):
+                o = hs.draft_step(st, u)
+                if j < N_D:
+                    S.append(o.argmax_ids[0])
+                    u = S[-1]
+            o = hs.verify_intermediate(st, S, N_D + 1)
+            Vh, _ = orc.leading_substring_verify(S, o.argmax_ids)
+            V += Vh
+            pending = V[-1]
+        o = hs.verify_target(st, V, len(V))
+        F, _ = orc.leading_substring_verify(V, o.argmax_ids)
+        pending = F[-1]
+        committed += len(F)
+        times.append(time.perf_counter() - t0)
+    total = sum(times)
+    return {"value": committed / total, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{budget_steps} super-round(s) of the same shape (2 x (6 draft steps + verify-I of 6 rows) + "
+                      f"verify-T) from a synthetic cached state of 1024 positions; {total:.1f} s of CPU work",
+            "s_per_step": total / budget_steps}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    from paper_2510_01336_b200 import workload as wl
+    shape = wl.L3_8B
+    # sized so that the whole run stays within a few minutes: one super-round per step, at most 3 timed steps
+    n = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    base = cpu_super_round(shape, None, budget_steps=n)
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": world,
+            "steps": n, "warmup": 0, "ms_per_step": base["s_per_step"] * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "configs[1] shape; the CPU oracle on a bounded sample", "requested_steps": args.steps,
+                       "wall_s": round(time.perf_counter() - t0, 1)},
+            "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

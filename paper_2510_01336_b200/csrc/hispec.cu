@@ -1,0 +1,609 @@
+// C ABI of the HiSpec verification library: context, argument checks and the launch
+// sequence of one stage call (steps a0..a10: row fetch, per layer [RMSNorm, QKV, RoPE + KV
+// append, paged causal attention, O + residual, RMSNorm, SwiGLU, down + residual], exit rows,
+// exit head + argmax, prefix acceptance + prune).
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+using namespace hispec;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][K] row-major, box = 64 (k) x box_rows, 128-byte swizzle, OOB reads give 0
+bool encode_2d(CUtensorMap *tm, const void *base, uint64_t K, uint64_t rows, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTileK, box_rows};
+    cuuint32_t es[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// activation buffer [2 planes][T_alloc][K]
+bool encode_act(CUtensorMap *tm, const void *base, uint64_t K, uint64_t T_alloc, uint32_t t_box, uint32_t planes) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {K, T_alloc, 2};
+    cuuint64_t strides[2] = {K * 2, T_alloc * K * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kTileK, t_box, planes};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int env_int(const char *name, int dflt) {
+    const char *s = getenv(name);
+    return (s && *s) ? atoi(s) : dflt;
+}
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
+
+struct ActMapCache {
+    const void *base;
+    int t_box, planes;
+    CUtensorMap map;
+};
+
+}  // namespace
+
+struct ProfEvent {
+    cudaEvent_t a, b;
+    int kind;
+    double bytes;
+};
+
+struct hispec_ctx_ext {
+    bool profiling;
+    std::vector<ProfEvent> *prof;       // recorded since the last read
+    std::vector<ProfEvent> *prof_free;  // event pairs ready for reuse
+    ActMapCache act_cache[3][8];
+    int act_cache_n[3];
+    int T_alloc;
+    int gemm_smem_budget;
+    bool pdl;
+};
+
+static hispec_ctx_ext *ext_of(hispec_ctx *c);
+
+struct hispec_ctx_full : hispec_ctx {
+    hispec_ctx_ext ext;
+};
+static hispec_ctx_ext *ext_of(hispec_ctx *c) { return &static_cast<hispec_ctx_full *>(c)->ext; }
+
+template <typename... KArgs, typename... Args>
+static cudaError_t launch(hispec_ctx *c, cudaStream_t st, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                          Args &&...args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ext_of(c)->pdl ? 1 : 0;
+    c->launches++;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+// event pair around one launch while profiling is on
+struct ProfScope {
+    hispec_ctx *c;
+    cudaStream_t st;
+    ProfEvent ev;
+    bool on;
+    ProfScope(hispec_ctx *c_, cudaStream_t st_, int kind, double bytes) : c(c_), st(st_), on(ext_of(c_)->profiling) {
+        if (!on) return;
+        hispec_ctx_ext *x = ext_of(c);
+        if (!x->prof_free->empty()) {
+            ev = x->prof_free->back();
+            x->prof_free->pop_back();
+        } else if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) {
+            on = false;
+            return;
+        }
+        ev.kind = kind;
+        ev.bytes = bytes;
+        cudaEventRecord(ev.a, st);
+    }
+    ~ProfScope() {
+        if (!on) return;
+        cudaEventRecord(ev.b, st);
+        ext_of(c)->prof->push_back(ev);
+    }
+};
+
+#define CK(expr)                              \
+    do {                                      \
+        cudaError_t e_ = (expr);              \
+        if (e_ != cudaSuccess) return HISPEC_ECUDA; \
+    } while (0)
+
+extern "C" const char *hispec_strerror(int code) {
+    switch (code) {
+        case HISPEC_OK: return "ok";
+        case HISPEC_EINVAL: return "invalid argument";
+        case HISPEC_ECAPACITY: return "request exceeds the context's capacity";
+        case HISPEC_ECUDA: return "CUDA call failed";
+        case HISPEC_ENOMEM: return "workspace allocation failed";
+        default: return "unknown error";
+    }
+}
+
+extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights *w, hispec_ctx **out) {
+    if (!desc || !w || !out) return HISPEC_EINVAL;
+    const hispec_model_desc &d = *desc;
+    if (d.n_layers <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.d_ffn <= 0 || d.vocab <= 0 ||
+        d.page_size <= 0 || d.max_batch <= 0 || d.max_rows_per_seq <= 0 || d.max_pages_per_seq <= 0)
+        return HISPEC_EINVAL;
+    if (d.n_q_heads % d.n_kv_heads) return HISPEC_EINVAL;
+    if (d.head_dim != 64 && d.head_dim != 128) return HISPEC_EINVAL;
+    if (d.d_model % 8 || d.d_ffn % 8) return HISPEC_EINVAL;  // TMA: 16-byte row pitch
+    if (d.max_rows_per_seq > kAttnMaxRows) return HISPEC_ECAPACITY;
+    if (!w->tok_emb || !w->wqkv || !w->wo || !w->wgu || !w->wdown || !w->attn_norm || !w->ffn_norm || !w->final_norm)
+        return HISPEC_EINVAL;
+
+    hispec_ctx_full *c = new (std::nothrow) hispec_ctx_full();
+    if (!c) return HISPEC_ENOMEM;
+    memset(static_cast<hispec_ctx *>(c), 0, sizeof(hispec_ctx));
+    memset(&c->ext, 0, sizeof(c->ext));
+    c->ext.prof = new std::vector<ProfEvent>();
+    c->ext.prof_free = new std::vector<ProfEvent>();
+    c->d = d;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return HISPEC_ECUDA; }
+    cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (c->sm_count <= 0) c->sm_count = 148;
+    const int L = d.n_layers;
+    c->tok_emb = w->tok_emb;
+    c->final_norm = w->final_norm;
+    c->wqkv = new const void *[L]; c->wo = new const void *[L]; c->wgu = new const void *[L]; c->wdown = new const void *[L];
+    c->attn_norm = new const float *[L]; c->ffn_norm = new const float *[L];
+    c->tm_wqkv = new CUtensorMap[L]; c->tm_wo = new CUtensorMap[L]; c->tm_wgu = new CUtensorMap[L]; c->tm_wdown = new CUtensorMap[L];
+    const int nq = d.n_q_heads * d.head_dim, nqkv = (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
+    bool simt = (d.flags & HISPEC_FLAG_SIMT_GEMM) != 0;
+    bool ok = true;
+    for (int l = 0; l < L; ++l) {
+        c->wqkv[l] = w->wqkv[l]; c->wo[l] = w->wo[l]; c->wgu[l] = w->wgu[l]; c->wdown[l] = w->wdown[l];
+        c->attn_norm[l] = w->attn_norm[l]; c->ffn_norm[l] = w->ffn_norm[l];
+        if (!simt && c->wqkv[l]) {
+            ok = ok && encode_2d(&c->tm_wqkv[l], c->wqkv[l], d.d_model, nqkv, kWeightTileRows);
+            ok = ok && encode_2d(&c->tm_wo[l], c->wo[l], nq, d.d_model, kWeightTileRows);
+            ok = ok && encode_2d(&c->tm_wgu[l], c->wgu[l], d.d_model, 2 * (uint64_t)d.d_ffn, kWeightTileRows);
+            ok = ok && encode_2d(&c->tm_wdown[l], c->wdown[l], d.d_ffn, d.d_model, kWeightTileRows);
+        }
+    }
+    if (!ok) { hispec_destroy(c); return HISPEC_ECUDA; }
+
+    // split-K plan: enough CTAs to put every SM to work on each projection
+    const int target = env_int("HISPEC_SPLIT_TARGET", c->sm_count);
+    auto plan = [&](GemmKind k, int N, int K, bool allow_split) {
+        GemmPlan &p = c->plan[k];
+        p.N = N; p.K = K; p.tiles = ceil_div(N, kWeightTileRows); p.kb_total = ceil_div(K, kTileK);
+        int s = allow_split ? target / p.tiles : 1;
+        if (s < 1) s = 1;
+        if (s > kMaxSplits) s = kMaxSplits;
+        if (s > p.kb_total) s = p.kb_total;
+        p.splits = s;
+    };
+    plan(G_QKV, nqkv, d.d_model, true);
+    plan(G_O, d.d_model, nq, true);
+    plan(G_GU, 2 * d.d_ffn, d.d_model, true);
+    plan(G_DOWN, d.d_model, d.d_ffn, true);
+    plan(G_HEAD, d.vocab, d.d_model, false);
+
+    c->T_max = d.max_batch * d.max_rows_per_seq;
+    const int T_alloc = round_up(c->T_max, 16);
+    c->ext.T_alloc = T_alloc;
+    c->ext.gemm_smem_budget = env_int("HISPEC_GEMM_SMEM", 100 * 1024);
+    c->ext.pdl = !(d.flags & HISPEC_FLAG_NO_PDL);
+    size_t part_floats = 0;
+    for (int k = 0; k < G_HEAD; ++k) {
+        size_t f = (size_t)c->plan[k].splits * T_alloc * c->plan[k].N;
+        if (f > part_floats) part_floats = f;
+    }
+    c->part_floats = part_floats;
+    c->attn_max_splits = 1;
+    auto alloc = [&](void **p, size_t bytes) { return cudaMalloc(p, bytes ? bytes : 16) == cudaSuccess; };
+    ok = true;
+    ok = ok && alloc((void **)&c->x, sizeof(float) * T_alloc * d.d_model);
+    ok = ok && alloc((void **)&c->act_d, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_model);
+    ok = ok && alloc((void **)&c->act_o, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * nq);
+    ok = ok && alloc((void **)&c->act_f, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_ffn);
+    ok = ok && alloc((void **)&c->q, sizeof(float) * (size_t)T_alloc * nq);
+    ok = ok && alloc((void **)&c->part, sizeof(float) * part_floats);
+    ok = ok && alloc((void **)&c->top_part, sizeof(float) * 4 * (size_t)c->plan[G_HEAD].tiles * 4 * T_alloc);
+    if (simt) ok = ok && alloc((void **)&c->logits_ws, sizeof(float) * (size_t)T_alloc * d.vocab);
+    ok = ok && alloc((void **)&c->inv_freq, sizeof(double) * (d.head_dim / 2));
+    ok = ok && alloc((void **)&c->rows.p0, sizeof(int32_t) * d.max_batch);
+    ok = ok && alloc((void **)&c->rows.n_rows, sizeof(int32_t) * d.max_batch);
+    ok = ok && alloc((void **)&c->rows.n_draft, sizeof(int32_t) * d.max_batch);
+    ok = ok && alloc((void **)&c->rows.dst_row, sizeof(int32_t) * d.max_batch);
+    ok = ok && alloc((void **)&c->argmax_ws, sizeof(int32_t) * T_alloc);
+    ok = ok && alloc((void **)&c->status, sizeof(uint32_t));
+    if (!ok) { hispec_destroy(c); return HISPEC_ENOMEM; }
+    bool e = true;
+    e = e && cudaMemset(c->status, 0, sizeof(uint32_t)) == cudaSuccess;
+    e = e && cudaMemset(c->act_d, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_model) == cudaSuccess;
+    e = e && cudaMemset(c->act_o, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * nq) == cudaSuccess;
+    e = e && cudaMemset(c->act_f, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_ffn) == cudaSuccess;
+    // rotary frequencies base^(-2i/hd) in double precision
+    int half = d.head_dim / 2;
+    double *f = new double[half];
+    for (int i = 0; i < half; ++i) f[i] = pow((double)d.rope_base, -2.0 * (double)i / (double)d.head_dim);
+    e = e && cudaMemcpy(c->inv_freq, f, sizeof(double) * half, cudaMemcpyHostToDevice) == cudaSuccess;
+    delete[] f;
+    e = e && cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+    if (!e) { hispec_destroy(c); return HISPEC_ECUDA; }
+    *out = c;
+    return HISPEC_OK;
+}
+
+extern "C" int hispec_destroy(hispec_ctx *c0) {
+    if (!c0) return HISPEC_EINVAL;
+    hispec_ctx_full *c = static_cast<hispec_ctx_full *>(c0);
+    void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->top_part, c->logits_ws, c->inv_freq,
+                    c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status};
+    for (void *p : bufs)
+        if (p) cudaFree(p);
+    delete[] c->wqkv; delete[] c->wo; delete[] c->wgu; delete[] c->wdown; delete[] c->attn_norm; delete[] c->ffn_norm;
+    delete[] c->tm_wqkv; delete[] c->tm_wo; delete[] c->tm_wgu; delete[] c->tm_wdown;
+    for (std::vector<ProfEvent> *v : {c->ext.prof, c->ext.prof_free})
+        if (v) {
+            for (ProfEvent &e : *v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+            delete v;
+        }
+    delete c;
+    return HISPEC_OK;
+}
+
+extern "C" int hispec_profile_enable(hispec_ctx *c, int on) {
+    if (!c) return HISPEC_EINVAL;
+    ext_of(c)->profiling = on != 0;
+    return HISPEC_OK;
+}
+
+extern "C" int hispec_profile_read(hispec_ctx *c, void *stream, int kind, double *ms, double *bytes, int64_t *launches) {
+    if (!c || !ms || !bytes || !launches) return HISPEC_EINVAL;
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    hispec_ctx_ext *x = ext_of(c);
+    double t = 0.0, by = 0.0;
+    int64_t n = 0;
+    std::vector<ProfEvent> keep;
+    for (ProfEvent &e : *x->prof) {
+        if (e.kind != kind) { keep.push_back(e); continue; }
+        float f = 0.0f;
+        if (cudaEventElapsedTime(&f, e.a, e.b) == cudaSuccess) { t += f; by += e.bytes; ++n; }
+        x->prof_free->push_back(e);
+    }
+    x->prof->swap(keep);
+    *ms = t; *bytes = by; *launches = n;
+    return HISPEC_OK;
+}
+
+extern "C" int64_t hispec_launch_count(const hispec_ctx *c) { return c ? c->launches : 0; }
+
+extern "C" int hispec_device_status(hispec_ctx *c, void *stream, uint32_t *host_out) {
+    if (!c || !host_out) return HISPEC_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    CK(cudaStreamSynchronize(st));
+    CK(cudaMemcpyAsync(host_out, c->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaMemsetAsync(c->status, 0, sizeof(uint32_t), st));
+    CK(cudaStreamSynchronize(st));
+    return HISPEC_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+const CUtensorMap *act_map(hispec_ctx *c, int which, const void *base, int K, int t_box, int planes) {
+    hispec_ctx_ext *x = ext_of(c);
+    for (int i = 0; i < x->act_cache_n[which]; ++i) {
+        ActMapCache &m = x->act_cache[which][i];
+        if (m.base == base && m.t_box == t_box && m.planes == planes) return &m.map;
+    }
+    int slot = x->act_cache_n[which] < 8 ? x->act_cache_n[which]++ : 7;
+    ActMapCache &m = x->act_cache[which][slot];
+    if (!encode_act(&m.map, base, K, x->T_alloc, t_box, planes)) return nullptr;
+    m.base = base; m.t_box = t_box; m.planes = planes;
+    return &m.map;
+}
+
+const CUtensorMap *head_map(hispec_ctx *c, const void *head) {
+    for (int i = 0; i < c->n_head_maps; ++i)
+        if (c->head_maps[i].ptr == head) return &c->head_maps[i].map;
+    int slot = c->n_head_maps < 4 ? c->n_head_maps++ : 3;
+    if (!encode_2d(&c->head_maps[slot].map, head, c->d.d_model, c->d.vocab, kWeightTileRows)) return nullptr;
+    c->head_maps[slot].ptr = head;
+    return &c->head_maps[slot].map;
+}
+
+struct StageCall {
+    StageArgs a;
+    const hispec_exits *exits;
+    const hispec_kv *kv;
+    const hispec_hidden *hidden;
+    const int32_t *tokens;     // embedding mode
+    const int32_t *n_tokens;   // prefill
+    const int32_t *draft_tokens, *n_draft, *n_rows;
+    int token_stride, out_stride;
+    const hispec_result *res;
+    int32_t *out_tokens;
+};
+
+// one projection: activation buffer `which` (0: act_d, 1: act_o, 2: act_f) times weight matrix
+int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const CUtensorMap *tmW, int which,
+             int T_pad, const StageCall &sc) {
+    const GemmPlan &p = c->plan[kind];
+    hispec_ctx_ext *x = ext_of(c);
+    const bool plain = (c->d.flags & HISPEC_FLAG_PLAIN_ACT) != 0;
+    const bool simt = (c->d.flags & HISPEC_FLAG_SIMT_GEMM) != 0;
+    const int planes = plain ? 1 : 2;
+    const __nv_bfloat16 *act = which == 0 ? c->act_d : (which == 1 ? c->act_o : c->act_f);
+    const bool head = kind == G_HEAD;
+    const size_t split_stride = (size_t)T_pad * p.N;
+    if (!head && (size_t)p.splits * split_stride > c->part_floats) return HISPEC_ECAPACITY;
+    const int chunk = planes == 2 ? 128 : 256;
+    for (int row0 = 0; row0 < T_pad; row0 += chunk) {
+        int rows = T_pad - row0 < chunk ? T_pad - row0 : chunk;
+        ProfScope prof(c, st, 0, 2.0 * (double)p.N * (double)p.K);
+        if (simt) {
+            float *outp = head ? c->logits_ws : c->part;
+            dim3 grid(ceil_div(p.N * 32, 256), head ? 1 : p.splits);
+            CK(launch(c, st, gemm_simt_kernel, grid, dim3(256), 0, (const __nv_bfloat16 *)W, act, x->T_alloc, planes, p.N,
+                      p.K, row0, rows, p.kb_total, head ? 1 : p.splits, outp, split_stride, p.N));
+            if (head) {
+                CK(launch(c, st, logits_tile_top2_kernel, dim3(p.tiles, rows), dim3(32), 0, (const float *)c->logits_ws,
+                          p.N, row0, rows, T_pad, c->top_part));
+                if (sc.res && sc.res->logits)
+                    CK(launch(c, st, copy_logits_kernel, dim3(ceil_div(p.N, 256), rows), dim3(256), 0, sc.a, c->rows,
+                              (const float *)c->logits_ws, p.N, row0, rows, sc.res->logits));
+            }
+            continue;
+        }
+        GemmArgs g;
+        memset(&g, 0, sizeof(g));
+        g.N = p.N; g.K = p.K; g.kb_total = p.kb_total; g.splits = head ? 1 : p.splits;
+        g.row0 = row0; g.rows = rows;
+        g.planes = planes;
+        g.t_box = round_up(rows, planes == 2 ? 8 : 16);
+        int ncols = g.t_box * planes;
+        int tc = 32;
+        while (tc < ncols) tc <<= 1;
+        g.tmem_cols = tc;
+        int stage_bytes = kWTileBytes + ncols * 128;
+        int stages = x->gemm_smem_budget / stage_bytes;
+        if (stages < 2) stages = 2;
+        if (stages > 16) stages = 16;
+        g.stages = stages;
+        g.head = head ? 1 : 0;
+        g.part = c->part; g.split_stride = split_stride;
+        g.top_part = c->top_part; g.T_pad = T_pad;
+        g.logits = (head && sc.res) ? sc.res->logits : nullptr;
+        g.R_pad = sc.a.R_pad; g.max_rows = sc.a.max_rows; g.n_rows = c->rows.n_rows;
+        g.status = c->status;
+        const CUtensorMap *tmX = act_map(c, which, act, p.K, g.t_box, planes);
+        if (!tmX || !tmW) return HISPEC_ECUDA;
+        size_t smem = (size_t)stages * stage_bytes + 1024;
+        CK(launch(c, st, gemm_tc_kernel, dim3(p.tiles, g.splits), dim3(kGemmThreads), smem, *tmW, *tmX, g));
+    }
+    return HISPEC_OK;
+}
+
+int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
+    const hispec_model_desc &d = c->d;
+    const StageArgs &a = sc.a;
+    hispec_ctx_ext *x = ext_of(c);
+    const int T_pad = a.batch * a.R_pad;
+    const int plain = (d.flags & HISPEC_FLAG_PLAIN_ACT) ? 1 : 0;
+    const bool simt = (d.flags & HISPEC_FLAG_SIMT_GEMM) != 0;
+    const hispec_kv &kv = *sc.kv;
+
+    CK(launch(c, st, prep_rows_kernel, dim3(ceil_div(a.batch, 64)), dim3(64), 0, a, (const int32_t *)kv.len_draft,
+              (const int32_t *)kv.len_inter, (const int32_t *)kv.len_target, sc.n_rows, sc.n_draft, sc.tokens,
+              sc.n_tokens, c->rows, c->status));
+    const float *h_src = nullptr;
+    if (a.mode == 1) h_src = (a.l0 == a.L_d) ? sc.hidden->h_draft : sc.hidden->h_inter;
+    CK(launch(c, st, rows_in_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, sc.tokens,
+              (const __nv_bfloat16 *)c->tok_emb, d.vocab, h_src, c->attn_norm[a.l0], d.rms_eps, d.d_model, c->x,
+              c->act_d, x->T_alloc, plain, c->status));
+
+    float *exit_buf = nullptr;
+    if (a.l1 == a.L_d) exit_buf = sc.hidden ? sc.hidden->h_draft : nullptr;
+    else if (a.l1 == a.L_i) exit_buf = sc.hidden ? sc.hidden->h_inter : nullptr;
+    float *hidden_out = sc.res ? sc.res->hidden_out : nullptr;
+
+    for (int l = a.l0; l < a.l1; ++l) {
+        const int pool_layer = l - kv.first_layer;
+        int rc;
+        const GemmPlan &pq = c->plan[G_QKV], &po = c->plan[G_O], &pg = c->plan[G_GU], &pd = c->plan[G_DOWN];
+        int sq = simt ? pq.splits : pq.splits;
+        if ((rc = run_gemm(c, st, G_QKV, c->wqkv[l], &c->tm_wqkv[l], 0, T_pad, sc)) != 0) return rc;
+        CK(launch(c, st, qkv_rope_store_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, sq,
+                  (size_t)T_pad * pq.N, d.n_q_heads, d.n_kv_heads, d.head_dim, (const double *)c->inv_freq, c->q,
+                  (__nv_bfloat16 *)kv.k_pages, (__nv_bfloat16 *)kv.v_pages, kv.block_table, (long long)kv.n_pages,
+                  pool_layer, c->status));
+        AttnArgs at;
+        at.q = c->q; at.k_pages = (const __nv_bfloat16 *)kv.k_pages; at.v_pages = (const __nv_bfloat16 *)kv.v_pages;
+        at.block_table = kv.block_table; at.n_pages = kv.n_pages; at.pool_layer = pool_layer;
+        at.hq = d.n_q_heads; at.hkv = d.n_kv_heads; at.hd = d.head_dim;
+        at.scale = 1.0f / sqrtf((float)d.head_dim);
+        at.out = c->act_o; at.T_alloc = x->T_alloc; at.plain = plain;
+        {
+            ProfScope prof(c, st, 1, 0.0);
+            int warps = T_pad * d.n_q_heads;
+            dim3 grid(ceil_div(warps, 4));
+            if (d.head_dim == 64) CK(launch(c, st, attention_rowwarp_kernel<64>, grid, dim3(128), 0, a, c->rows, at, c->status));
+            else CK(launch(c, st, attention_rowwarp_kernel<128>, grid, dim3(128), 0, a, c->rows, at, c->status));
+        }
+        if ((rc = run_gemm(c, st, G_O, c->wo[l], &c->tm_wo[l], 1, T_pad, sc)) != 0) return rc;
+        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, po.splits,
+                  (size_t)T_pad * po.N, c->ffn_norm[l], d.rms_eps, d.d_model, c->x, c->act_d, x->T_alloc, plain,
+                  (float *)nullptr, (float *)nullptr));
+        if ((rc = run_gemm(c, st, G_GU, c->wgu[l], &c->tm_wgu[l], 0, T_pad, sc)) != 0) return rc;
+        CK(launch(c, st, silu_mul_kernel, dim3(ceil_div(d.d_ffn, 256), T_pad), dim3(256), 0, (const float *)c->part,
+                  pg.splits, (size_t)T_pad * pg.N, d.d_ffn, c->act_f, x->T_alloc, plain));
+        if ((rc = run_gemm(c, st, G_DOWN, c->wdown[l], &c->tm_wdown[l], 2, T_pad, sc)) != 0) return rc;
+        const bool last = (l + 1 == a.l1);
+        const float *gain = last ? c->final_norm : c->attn_norm[l + 1];
+        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, pd.splits,
+                  (size_t)T_pad * pd.N, gain, d.rms_eps, d.d_model, c->x, c->act_d, x->T_alloc, plain,
+                  last ? exit_buf : (float *)nullptr, last ? hidden_out : (float *)nullptr));
+    }
+    const void *head = (a.l1 == a.L_d) ? sc.exits->head_d : ((a.l1 == a.L_i) ? sc.exits->head_i : sc.exits->head_f);
+    const CUtensorMap *tmH = simt ? (const CUtensorMap *)c->tm_wqkv : head_map(c, head);
+    int rc = run_gemm(c, st, G_HEAD, head, tmH, 0, T_pad, sc);
+    if (rc) return rc;
+    AcceptArgs r;
+    memset(&r, 0, sizeof(r));
+    r.len_d = kv.len_draft; r.len_i = kv.len_inter; r.len_f = kv.len_target;
+    r.draft_tokens = sc.draft_tokens; r.token_stride = sc.token_stride; r.out_stride = sc.out_stride;
+    if (sc.res) {
+        r.n_accepted = sc.res->n_accepted; r.next_token = sc.res->next_token;
+        r.argmax_ids = sc.res->argmax_ids; r.top2 = sc.res->top2; r.tentative = sc.res->tentative;
+        r.pending = sc.res->pending;
+    }
+    r.out_tokens = sc.out_tokens;
+    r.n_tokens = sc.n_tokens;
+    int n_tiles = simt ? c->plan[G_HEAD].tiles : 4 * c->plan[G_HEAD].tiles;
+    CK(launch(c, st, head_reduce_accept_kernel, dim3(a.batch), dim3(256), 0, a, c->rows, (const float *)c->top_part,
+              n_tiles, T_pad, r, c->argmax_ws));
+    return HISPEC_OK;
+}
+
+int check_common(hispec_ctx *c, int l0, int l1, const hispec_exits *ex, const hispec_kv *kv, int batch) {
+    if (!c || !ex || !kv) return HISPEC_EINVAL;
+    if (!(0 < ex->L_d && ex->L_d < ex->L_i && ex->L_i < ex->L_f && ex->L_f <= c->d.n_layers)) return HISPEC_EINVAL;
+    if (l0 < 0 || l1 <= l0 || l1 > c->d.n_layers) return HISPEC_EINVAL;
+    if (l1 != ex->L_d && l1 != ex->L_i && l1 != ex->L_f) return HISPEC_EINVAL;
+    const void *head = (l1 == ex->L_d) ? ex->head_d : ((l1 == ex->L_i) ? ex->head_i : ex->head_f);
+    if (!head) return HISPEC_EINVAL;
+    if (batch <= 0) return HISPEC_EINVAL;
+    if (batch > c->d.max_batch) return HISPEC_ECAPACITY;
+    if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->len_draft || !kv->len_inter || !kv->len_target ||
+        kv->n_pages <= 0)
+        return HISPEC_EINVAL;
+    if (kv->first_layer < 0 || l0 < kv->first_layer || l1 > kv->first_layer + kv->n_pool_layers) return HISPEC_EINVAL;
+    for (int l = l0; l < l1; ++l)
+        if (!c->wqkv[l] || !c->wo[l] || !c->wgu[l] || !c->wdown[l] || !c->attn_norm[l] || !c->ffn_norm[l])
+            return HISPEC_EINVAL;
+    return HISPEC_OK;
+}
+
+StageArgs base_args(hispec_ctx *c, const hispec_exits *ex, int l0, int l1, int batch, int R_pad) {
+    StageArgs a;
+    memset(&a, 0, sizeof(a));
+    a.L_d = ex->L_d; a.L_i = ex->L_i; a.L_f = ex->L_f; a.l0 = l0; a.l1 = l1;
+    a.batch = batch; a.R_pad = R_pad; a.max_rows = c->d.max_rows_per_seq; a.max_pages = c->d.max_pages_per_seq;
+    a.page_size = c->d.page_size;
+    return a;
+}
+
+int verify_call(hispec_ctx *c, void *stream, int l0, int l1, const hispec_exits *ex, const hispec_kv *kv,
+                const hispec_hidden *hid, int batch, const int32_t *draft_tokens, int token_stride,
+                const int32_t *n_draft, const int32_t *n_rows, int k, const hispec_result *res, bool target) {
+    int rc = check_common(c, l0, l1, ex, kv, batch);
+    if (rc) return rc;
+    if (!hid || !hid->h_draft || !hid->h_inter || !draft_tokens || !res || !res->n_accepted || !res->next_token)
+        return HISPEC_EINVAL;
+    if ((n_draft == nullptr) != (n_rows == nullptr)) return HISPEC_EINVAL;
+    if (k < 0 || token_stride < k) return HISPEC_EINVAL;
+    if (k + 1 > c->d.max_rows_per_seq) return HISPEC_ECAPACITY;
+    if (target) {
+        if (l0 != ex->L_i || l1 != ex->L_f) return HISPEC_EINVAL;
+    } else {
+        if (l0 != ex->L_d || (l1 != ex->L_i && l1 != ex->L_f)) return HISPEC_EINVAL;
+    }
+    StageCall sc;
+    memset(&sc, 0, sizeof(sc));
+    sc.a = base_args(c, ex, l0, l1, batch, k + 1);
+    sc.a.mode = 1; sc.a.k = k; sc.a.is_target = target ? 1 : 0;
+    sc.exits = ex; sc.kv = kv; sc.hidden = hid;
+    sc.draft_tokens = draft_tokens; sc.n_draft = n_draft; sc.n_rows = n_rows; sc.token_stride = token_stride;
+    sc.res = res;
+    return run_stage(c, (cudaStream_t)stream, sc);
+}
+
+}  // namespace
+
+extern "C" int hispec_draft(hispec_ctx *c, void *stream, int l0, int l1, const hispec_exits *ex, const hispec_kv *kv,
+                            const hispec_hidden *hid, int batch, const int32_t *in_tokens, int in_stride,
+                            int32_t *out_tokens, int out_stride, const hispec_result *res) {
+    int rc = check_common(c, l0, l1, ex, kv, batch);
+    if (rc) return rc;
+    if (l0 != 0 || !in_tokens || in_stride < 1 || (out_tokens && out_stride < 1)) return HISPEC_EINVAL;
+    if (l1 != ex->L_f && (!hid || !hid->h_draft || !hid->h_inter)) return HISPEC_EINVAL;
+    StageCall sc;
+    memset(&sc, 0, sizeof(sc));
+    sc.a = base_args(c, ex, l0, l1, batch, 1);
+    sc.a.mode = 0; sc.a.tok_stride = in_stride; sc.a.tok_offset = 0; sc.a.fixed_rows = 1;
+    sc.exits = ex; sc.kv = kv; sc.hidden = hid; sc.tokens = in_tokens; sc.res = res; sc.out_tokens = out_tokens;
+    sc.out_stride = out_stride;
+    return run_stage(c, (cudaStream_t)stream, sc);
+}
+
+extern "C" int hispec_verify_intermediate(hispec_ctx *c, void *stream, int l0, int l1, const hispec_exits *ex,
+                                          const hispec_kv *kv, const hispec_hidden *hid, int batch,
+                                          const int32_t *draft_tokens, int token_stride, const int32_t *n_draft,
+                                          const int32_t *n_rows, int k, const hispec_result *res) {
+    return verify_call(c, stream, l0, l1, ex, kv, hid, batch, draft_tokens, token_stride, n_draft, n_rows, k, res, false);
+}
+
+extern "C" int hispec_verify_target(hispec_ctx *c, void *stream, int l0, int l1, const hispec_exits *ex,
+                                    const hispec_kv *kv, const hispec_hidden *hid, int batch,
+                                    const int32_t *draft_tokens, int token_stride, const int32_t *n_draft,
+                                    const int32_t *n_rows, int k, const hispec_result *res) {
+    return verify_call(c, stream, l0, l1, ex, kv, hid, batch, draft_tokens, token_stride, n_draft, n_rows, k, res, true);
+}
+
+extern "C" int hispec_prefill(hispec_ctx *c, void *stream, const hispec_exits *ex, const hispec_kv *kv, int batch,
+                              const int32_t *tokens, const int32_t *n_tokens, int max_tokens, int32_t *first_token) {
+    if (!ex) return HISPEC_EINVAL;
+    int rc = check_common(c, 0, ex->L_f, ex, kv, batch);
+    if (rc) return rc;
+    if (!tokens || !n_tokens || max_tokens <= 0) return HISPEC_EINVAL;
+    const int C = c->d.max_rows_per_seq;
+    for (int off = 0; off < max_tokens; off += C) {
+        StageCall sc;
+        memset(&sc, 0, sizeof(sc));
+        sc.a = base_args(c, ex, 0, ex->L_f, batch, C);
+        sc.a.mode = 0; sc.a.tok_stride = max_tokens; sc.a.tok_offset = off;
+        sc.exits = ex; sc.kv = kv; sc.tokens = tokens; sc.n_tokens = n_tokens; sc.out_tokens = first_token;
+        sc.out_stride = 1;
+        rc = run_stage(c, (cudaStream_t)stream, sc);
+        if (rc) return rc;
+    }
+    return HISPEC_OK;
+}

@@ -1,0 +1,164 @@
+"""Host decoding loops over the C-ABI calls: HiSpec (Algorithm 2), single-stage
+self-speculation (Algorithm 1) and plain auto-regressive decoding.
+
+The loops only sequence calls and keep token lists; all arithmetic, the
+acceptance rule and the pruning of the shared state run in the library's
+kernels.  A super-round of HiSpec (m rounds of [N_d (+1) draft steps,
+intermediate verification] followed by one target verification) is enqueued
+without any host synchronisation: draft ids flow from one draft step to the
+next and into the verifier through device memory, the list V of tentatively
+accepted tokens is assembled by the intermediate verifier's acceptance kernel,
+and the target verifier takes its row count from the length counters.  The
+host reads back one small record per super-round.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Callable, List, Optional
+
+import torch
+
+from . import binding
+
+
+@dataclass
+class LoopStats:
+    super_rounds: int = 0
+    draft_steps: int = 0
+    inter_calls: int = 0
+    target_calls: int = 0
+    inter_accepted: int = 0
+    target_checked: int = 0
+    target_accepted: int = 0
+    committed: int = 0
+
+
+class HiSpecLoop:
+    """Batch of sequences decoded in lockstep (every sequence runs the same phase; the
+    acceptance outcome is per sequence)."""
+
+    def __init__(self, ctx: binding.Context, st: binding.KVState, batch: int, N_d: int, rounds: int = 2,
+                 bonus_inter: bool = True, device: str = "cuda"):
+        per_round = N_d + (1 if bonus_inter else 0)
+        assert per_round * rounds <= ctx.max_rows - 1, "hidden buffers too small: need rounds * (N_d + 1) + 1 rows"
+        self.ctx, self.st, self.B, self.N_d, self.rounds, self.bonus = ctx, st, batch, N_d, rounds, bonus_inter
+        i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device=device)
+        self.pending = i32(batch)                      # token waiting to enter the draft layers
+        self.S = i32(batch, N_d)                       # draft block of the current round
+        self.res_i = [binding.Result(i32(batch), i32(batch)) for _ in range(rounds)]
+        self.V = i32(batch, ctx.max_rows)              # tentatively accepted tokens (device-assembled)
+        for r in self.res_i:
+            r.tentative = self.V
+            r.pending = self.pending
+        self.res_t = binding.Result(i32(batch), i32(batch))
+        self.res_t.pending = self.pending
+        self.len_snapshot = i32(batch)
+        # pinned host mirrors read once per super-round
+        self.h_acc = torch.zeros(batch, dtype=torch.int32).pin_memory()
+        self.h_next = torch.zeros(batch, dtype=torch.int32).pin_memory()
+        self.h_V = torch.zeros((batch, ctx.max_rows), dtype=torch.int32).pin_memory()
+        self.h_acc_i = torch.zeros((rounds, batch), dtype=torch.int32).pin_memory()
+        self.h_nv = torch.zeros(batch, dtype=torch.int32).pin_memory()
+        self.stats = LoopStats()
+        self.tokens: List[List[int]] = [[] for _ in range(batch)]
+
+    # -- prompt ---------------------------------------------------------------------------
+    def prefill(self, prompts: List[List[int]]):
+        B = self.B
+        mx = max(len(p) for p in prompts)
+        toks = torch.zeros((B, mx), dtype=torch.int32)
+        for b, p in enumerate(prompts):
+            toks[b, : len(p)] = torch.tensor(p, dtype=torch.int32)
+        n = torch.tensor([len(p) for p in prompts], dtype=torch.int32)
+        self.ctx.prefill(self.st, toks.cuda(), n.cuda(), self.pending)
+        torch.cuda.synchronize()
+        first = self.pending.cpu().tolist()
+        for b in range(B):
+            self.tokens[b] = [first[b]]
+        return first
+
+    # -- one super-round, enqueued without host synchronisation ---------------------------------
+    def enqueue_super_round(self, stream=None):
+        ctx, st, N_d, B = self.ctx, self.st, self.N_d, self.B
+        S_ptr = self.S.data_ptr()
+        for r in range(self.rounds):
+            src = self.pending  # kept current by the acceptance kernel of the previous verification
+            # Generate(L_d, ., N_d): step j reads column j-1 of S (or the pending token) and writes column j
+            for j in range(N_d):
+                if j == 0:
+                    ctx.draft(st, src, S_ptr, batch=B, in_stride=1, out_stride=N_d, stream=stream)
+                else:
+                    ctx.draft(st, S_ptr + 4 * (j - 1), S_ptr + 4 * j, batch=B, in_stride=N_d, out_stride=N_d,
+                              stream=stream)
+            if self.bonus:  # push S_{N_d} through the draft layers so that L_i can emit v_{N_d+1}
+                ctx.draft(st, S_ptr + 4 * (N_d - 1), None, batch=B, in_stride=N_d, stream=stream)
+            ctx.verify_intermediate(st, self.S, None, None, self.res_i[r], stream=stream, k=N_d)
+            self.stats.draft_steps += N_d + (1 if self.bonus else 0)
+            self.stats.inter_calls += 1
+        # LeadingSubstringVerify(V, L_f, x): rows and |V| come from the length counters
+        ctx.verify_target(st, self.V, None, None, self.res_t, stream=stream, k=ctx.max_rows - 1)
+        self.stats.target_calls += 1
+        self.stats.super_rounds += 1
+
+    def collect(self, stream=None):
+        """Read back the outcome of the last super-round and extend the token lists.
+        Must follow enqueue_super_round; synchronises the stream."""
+        s = stream if stream is not None else torch.cuda.current_stream()
+        with torch.cuda.stream(s):
+            self.h_acc.copy_(self.res_t.n_accepted, non_blocking=True)
+            self.h_next.copy_(self.res_t.next_token, non_blocking=True)
+            self.h_V.copy_(self.V, non_blocking=True)
+            for r in range(self.rounds):
+                self.h_acc_i[r].copy_(self.res_i[r].n_accepted, non_blocking=True)
+        s.synchronize()
+        new = []
+        for b in range(self.B):
+            a = int(self.h_acc[b])
+            nxt = int(self.h_next[b])
+            F = self.h_V[b, :a].tolist() + ([nxt] if nxt >= 0 else [])
+            self.tokens[b] += F
+            new.append(F)
+            self.stats.target_accepted += a
+            self.stats.committed += len(F)
+            self.stats.inter_accepted += int(self.h_acc_i[:, b].sum())
+        return new
+
+    def generate(self, n_gen: int) -> List[List[int]]:
+        while min(len(t) for t in self.tokens) < n_gen:
+            self.enqueue_super_round()
+            self.collect()
+        return [t[:n_gen] for t in self.tokens]
+
+
+class ARLoop:
+    """Vanilla auto-regressive decoding: hispec_draft over [0, L_f) with the L_f exit, one row per step."""
+
+    def __init__(self, ctx: binding.Context, st: binding.KVState, batch: int, device: str = "cuda"):
+        self.ctx, self.st, self.B = ctx, st, batch
+        self.buf = [torch.zeros(batch, dtype=torch.int32, device=device) for _ in range(2)]
+        self.tokens: List[List[int]] = [[] for _ in range(batch)]
+
+    def prefill(self, prompts: List[List[int]]):
+        B = self.B
+        mx = max(len(p) for p in prompts)
+        toks = torch.zeros((B, mx), dtype=torch.int32)
+        for b, p in enumerate(prompts):
+            toks[b, : len(p)] = torch.tensor(p, dtype=torch.int32)
+        n = torch.tensor([len(p) for p in prompts], dtype=torch.int32)
+        self.ctx.prefill(self.st, toks.cuda(), n.cuda(), self.buf[0])
+        torch.cuda.synchronize()
+        first = self.buf[0].cpu().tolist()
+        self.tokens = [[t] for t in first]
+        return first
+
+    def generate(self, n_gen: int, stream=None) -> List[List[int]]:
+        hist = [self.buf[0].clone()]
+        cur = 0
+        for _ in range(n_gen - 1):
+            self.ctx.draft(self.st, self.buf[cur], self.buf[1 - cur], layer_end=self.ctx.exits.L_f, stream=stream)
+            cur = 1 - cur
+            hist.append(self.buf[cur].clone())
+        torch.cuda.synchronize()
+        allt = torch.stack(hist, 1).cpu().tolist()
+        self.tokens = [list(t) for t in allt]
+        return self.tokens

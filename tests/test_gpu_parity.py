@@ -1,0 +1,268 @@
+"""GPU parity: every C-ABI call against the oracle's stage call on the same seeded
+inputs, teacher-forced (the oracle's state is loaded before each call), through
+libhispec.so.  Tolerances: exit hidden rows 1e-2 relative L2, logits 5e-2 max
+abs, ids / accepted length / correction token bit-exact except where the
+oracle's top-2 margin is below 0.1 (there the id must lie in the near-tie set and
+the acceptance must follow the GPU's own ids)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.hispec import GenStats, HiSpecOracle, OracleModel
+from paper_2510_01336_b200 import workload as wl
+from tests import gpu_harness as gh
+from tests.helpers import oracle_for
+
+pytestmark = pytest.mark.gpu
+
+FLAG_SETS = {"tcgen05": 0, "simt": 1, "tcgen05-plain": 2}
+
+
+def _binding():
+    from paper_2510_01336_b200 import binding
+    return binding
+
+
+class GpuObserver:
+    """Runs every stage call of the oracle's decoding loop on the GPU as well, from the oracle's state."""
+
+    def __init__(self, ctx, st, hs, page_size, max_rows):
+        self.ctx, self.st, self.hs, self.ps, self.max_rows = ctx, st, hs, page_size, max_rows
+        self.layers = list(range(hs.m.n_layers))
+        self.calls = {"draft": 0, "verify_i": 0, "verify_t": 0}
+        self.worst = {"rel_l2": 0.0, "logit_err": 0.0, "exempt": 0, "rows": 0}
+        self.b = _binding()
+
+    def before(self, kind, ost, seq_tokens, **kw):
+        b = self.b
+        gh.load_seq(self.st, 0, ost, self.ps, self.layers, self.max_rows)
+        self.res = self.ctx.new_result(1, logits=True, hidden=True)
+        self.kind, self.kw = kind, kw
+        self.pre = (ost.len_d, ost.len_i, ost.len_f)
+        dev = "cuda"
+        if kind == "draft":
+            self.out_tok = torch.full((1,), -5, dtype=torch.int32, device=dev)
+            self.ctx.draft(self.st, torch.tensor([kw["token"]], dtype=torch.int32, device=dev), self.out_tok, self.res)
+        else:
+            S, R = kw["S"], kw["n_rows"]
+            k = max(len(S), 1)
+            dt = torch.zeros((1, k), dtype=torch.int32, device=dev)
+            if S:
+                dt[0, : len(S)] = torch.tensor(S, dtype=torch.int32)
+            nd = torch.tensor([len(S)], dtype=torch.int32, device=dev)
+            nr = torch.tensor([R], dtype=torch.int32, device=dev)
+            fn = self.ctx.verify_intermediate if kind == "verify_i" else self.ctx.verify_target
+            fn(self.st, dt, nd, nr, self.res)
+        torch.cuda.synchronize()
+        assert self.ctx.status() == 0
+
+    def after(self, kind, ost, out):
+        hs, st = self.hs, self.st
+        R = 1 if kind == "draft" else self.kw["n_rows"]
+        S = [] if kind == "draft" else self.kw["S"]
+        s = gh.compare_exit(out, self.res, 0, R, S, check_accept=(kind != "draft"), tag=f"{kind}#{self.calls[kind]}")
+        for k in ("rel_l2", "logit_err"):
+            self.worst[k] = max(self.worst[k], s[k])
+        self.worst["exempt"] += s["exempt"]
+        self.worst["rows"] += R
+        l0, l1, p0 = {"draft": (0, hs.L_d, self.pre[0]), "verify_i": (hs.L_d, hs.L_i, self.pre[1]),
+                      "verify_t": (hs.L_i, hs.L_f, self.pre[2])}[kind]
+        gh.compare_kv(st, 0, ost, self.ps, range(l0, l1), range(p0, p0 + R), tag=kind)
+        if kind == "draft":
+            gid = int(self.out_tok[0])
+            assert gid == int(self.res.argmax_ids[0, 0])
+            exp = (self.pre[0] + 1, self.pre[1], self.pre[2])
+            row = st.h_draft[0, self.pre[0] - self.pre[1]].cpu().numpy()
+            assert np.linalg.norm(row - out.hidden[0]) <= gh.HIDDEN_REL_L2 * np.linalg.norm(out.hidden[0])
+        else:
+            a = int(self.res.n_accepted[0])
+            nl = p0 + min(a + 1, R)
+            exp = (nl, nl, self.pre[2]) if kind == "verify_i" else (nl, nl, nl)
+            if kind == "verify_i":
+                base = self.pre[1] - self.pre[2]
+                rows = st.h_inter[0, base: base + R].cpu().numpy()
+                rel = np.linalg.norm(rows - out.hidden, axis=1) / np.linalg.norm(out.hidden, axis=1)
+                assert rel.max() <= gh.HIDDEN_REL_L2
+        got = (int(st.len_draft[0]), int(st.len_inter[0]), int(st.len_target[0]))
+        assert got == exp, f"{kind}: lengths {got} != {exp}"
+        self.calls[kind] += 1
+
+
+def _tiny_setup(flags, n_prompt, n_gen, N_d, rounds):
+    b = _binding()
+    shape = wl.TINY
+    w, m, hs = oracle_for(shape, kv_round=True)
+    max_rows = rounds * (N_d + 1) + 2
+    max_pages = (n_prompt + n_gen + max_rows + 2 + 15) // 16 + 1
+    ctx = b.Context(shape, w.to("cuda"), page_size=16, max_batch=1, max_rows_per_seq=max_rows,
+                    max_pages_per_seq=max_pages, flags=flags)
+    bt = wl.make_block_table(shape, 1, max_pages, n_pages=max_pages + 5)
+    st = ctx.new_state(1, max_pages + 5, bt)
+    return shape, w, m, hs, ctx, st, max_rows
+
+
+@pytest.mark.parametrize("flagname", ["simt", "tcgen05", "tcgen05-plain"])
+def test_tiny_config_every_call(flagname):
+    """cfg "tiny" as stated: prompt 128, k = 4 greedy drafts from the draft exit, target every 2
+    rounds, 64 generated tokens -- every draft / verify-I / verify-T call compared."""
+    n_gen = 64 if flagname == "tcgen05" else 12
+    shape, w, m, hs, ctx, st, max_rows = _tiny_setup(FLAG_SETS[flagname], 128, n_gen, 4, 2)
+    prompt = wl.make_tokens(shape, 128).tolist()
+    obs = GpuObserver(ctx, st, hs, 16, max_rows)
+    out = hs.hispec_generate(prompt, n_gen, 4, rounds=2, observer=obs, rows_cap=max_rows)
+    assert len(out) == n_gen and min(obs.calls.values()) > 0
+    print(f"\n[{flagname}] calls {obs.calls} worst rel-L2 {obs.worst['rel_l2']:.2e} logits {obs.worst['logit_err']:.2e} "
+          f"exempt rows {obs.worst['exempt']}/{obs.worst['rows']}")
+    ctx.close()
+
+
+def test_tiny_accepting_drafts_and_target_bonus():
+    """Drafts that the verifiers mostly accept (the target's greedy continuation, 25 % corrupted), the paper's
+    |V| >= N_i trigger and a bonus row at the target: accept, partial-accept and reject paths on the GPU."""
+    shape, w, m, hs, ctx, st, max_rows = _tiny_setup(0, 40, 30, 3, 3)
+    prompt = wl.make_tokens(shape, 40).tolist()
+    ar = hs.ar_generate(prompt, 50)
+    rng = np.random.default_rng(5)
+    override = lambda pos, g: ar[pos - len(prompt)] if (pos - len(prompt) < len(ar) and rng.random() < 0.75) else g
+    obs = GpuObserver(ctx, st, hs, 16, max_rows)
+    stt = GenStats()
+    out = hs.hispec_generate(prompt, 30, 3, N_i=4, bonus_target=True, draft_override=override, observer=obs,
+                             stats=stt, rows_cap=max_rows)
+    assert out == ar[:30] and stt.inter_accepted > 5 and stt.target_accepted > 5
+    ctx.close()
+
+
+def test_tiny_prefill_and_free_running_lossless():
+    """Prefill vs the oracle; then, free-running on the GPU alone, HiSpec's output must equal the GPU's own
+    auto-regressive greedy output (the lossless guarantee, on the device arithmetic)."""
+    b = _binding()
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecLoop
+    shape = wl.TINY
+    w, m, hs = oracle_for(shape, kv_round=True)
+    wg = w.to("cuda")
+    n_prompt, n_gen, N_d, rounds = 128, 64, 4, 2
+    max_rows = rounds * (N_d + 1) + 3
+    max_pages = (n_prompt + n_gen + 40) // 16 + 1
+    prompt = wl.make_tokens(shape, n_prompt).tolist()
+
+    ctx = b.Context(shape, wg, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    bt = wl.make_block_table(shape, 1, max_pages)
+    st = ctx.new_state(1, max_pages, bt)
+    loop = HiSpecLoop(ctx, st, 1, N_d, rounds)
+    first = loop.prefill([prompt])
+    # oracle prefill: first token (margin rule), lengths, KV of every layer
+    ost = hs.new_state(n_prompt + 8, 4)
+    o = hs.prefill(ost, prompt)
+    if o.top2[0, 0] - o.top2[0, 1] >= gh.MARGIN:
+        assert first[0] == o.argmax_ids[0]
+    assert (int(st.len_draft[0]), int(st.len_inter[0]), int(st.len_target[0])) == (n_prompt,) * 3
+    bt_row = st.block_table[0].cpu()
+    for l in range(shape.n_layers):
+        g = gh.cache_from_pages(st.k_pages, bt_row, 16, l, 0, range(n_prompt))
+        r = ost.cache.k[l, :n_prompt]
+        assert np.linalg.norm(g - r) / np.linalg.norm(r) < 1e-2
+    toks = loop.generate(n_gen)[0]
+    assert ctx.status() == 0
+
+    ctx2 = b.Context(shape, wg, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    st2 = ctx2.new_state(1, max_pages, bt)
+    ar = ARLoop(ctx2, st2, 1)
+    ar.prefill([prompt])
+    ar_toks = ar.generate(n_gen)[0]
+    assert ctx2.status() == 0
+    assert toks == ar_toks, "HiSpec on the GPU must reproduce the GPU's auto-regressive greedy output"
+    assert loop.stats.committed >= n_gen - 1 and loop.stats.target_calls > 0
+    ctx.close(); ctx2.close()
+
+
+@pytest.mark.parametrize("flagname", ["tcgen05", "simt"])
+def test_batched_ragged_gqa_pages_permuted(flagname):
+    """GQA 2:1, head_dim 128, odd sizes (d 320, ffn 400, vocab 1000): a batch of 3 sequences with different
+    context lengths, ragged row counts and scattered pages against the oracle, one sequence at a time;
+    then the same call with another page permutation must give bit-identical results."""
+    b = _binding()
+    shape = wl.MINI_GQA
+    w, m, hs = oracle_for(shape, kv_round=True)
+    B, N_d, max_rows, page = 3, 4, 8, 16
+    ctx_lens = [37, 5, 64]
+    n_rows = [5, 3, 4]
+    n_draft = [4, 3, 4]
+    max_pages = 8
+    ctx = b.Context(shape, w.to("cuda"), page_size=page, max_batch=B, max_rows_per_seq=max_rows,
+                    max_pages_per_seq=max_pages, flags=FLAG_SETS[flagname])
+    outs, states = [], []
+    drafts = []
+    for s in range(B):
+        prompt = wl.make_tokens(shape, ctx_lens[s], seed_offset=100 + s).tolist()
+        ost = hs.new_state(ctx_lens[s] + 16, max_rows)
+        pending = hs.prefill(ost, prompt).argmax_ids[0]
+        ar = hs.ar_generate(prompt, 8)
+        S = [ar[1 + j] if j < 2 else (ar[1 + j] + 7) % shape.vocab for j in range(n_draft[s])]
+        u = pending
+        for t in (S + [None])[: n_rows[s]]:
+            hs.draft_step(ost, u)
+            u = t
+        drafts.append(S)
+        states.append(ost)
+    results = []
+    for perm_seed in (3000, 3001):
+        bt = wl.make_block_table(shape, B, max_pages, n_pages=B * max_pages + 7, seed_offset=perm_seed)
+        st = ctx.new_state(B, B * max_pages + 7, bt)
+        for s in range(B):
+            gh.load_seq(st, s, states[s], page, range(shape.n_layers), max_rows)
+        res = ctx.new_result(B, logits=True, hidden=True)
+        dt = torch.zeros((B, N_d), dtype=torch.int32)
+        for s in range(B):
+            dt[s, : n_draft[s]] = torch.tensor(drafts[s], dtype=torch.int32)
+        ctx.verify_intermediate(st, dt.cuda(), torch.tensor(n_draft, dtype=torch.int32).cuda(),
+                                torch.tensor(n_rows, dtype=torch.int32).cuda(), res)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        results.append((res, st))
+    import copy
+    res, st = results[0]
+    for s in range(B):
+        ost = copy.deepcopy(states[s])
+        p0 = ost.len_i
+        out = hs.verify_intermediate(ost, drafts[s], n_rows[s])
+        gh.compare_exit(out, res, s, n_rows[s], drafts[s], check_accept=True, tag=f"seq{s}")
+        gh.compare_kv(st, s, ost, page, range(hs.L_d, hs.L_i), range(p0, p0 + n_rows[s]), tag=f"seq{s}")
+        assert int(st.len_inter[s]) == ost.len_i == int(st.len_draft[s])
+    r2 = results[1][0]
+    for name in ("n_accepted", "next_token", "argmax_ids", "logits", "hidden_out"):
+        assert torch.equal(getattr(res, name), getattr(r2, name)), f"page permutation changed {name}"
+    ctx.close()
+
+
+def test_errors_and_status_word():
+    """Host-detected errors return codes and enqueue nothing; device-detected faults set status bits and
+    the call completes (no trap, no hang)."""
+    b = _binding()
+    shape = wl.TINY
+    w = wl.make_weights(shape).to("cuda")
+    ctx = b.Context(shape, w, max_batch=2, max_rows_per_seq=6, max_pages_per_seq=4)
+    bt = wl.make_block_table(shape, 2, 4)
+    st = ctx.new_state(2, 8, bt)
+    res = ctx.new_result(2)
+    i32 = lambda v: torch.tensor(v, dtype=torch.int32, device="cuda")
+    dt = torch.zeros((2, 3), dtype=torch.int32, device="cuda")
+    with pytest.raises(b.HiSpecError):   # k + 1 rows exceed max_rows_per_seq
+        ctx.verify_intermediate(st, torch.zeros((2, 9), dtype=torch.int32, device="cuda"), i32([1, 1]), i32([1, 1]), res)
+    with pytest.raises(b.HiSpecError):   # layer_end is not an exit
+        ctx.draft(st, i32([1, 2]), layer_end=3)
+    with pytest.raises(b.HiSpecError):   # batch over capacity
+        ctx.draft(st, i32([1, 2, 3]))
+    n0 = ctx.launch_count()
+    # rows that were never buffered: STATE bit, lengths untouched
+    ctx.verify_intermediate(st, dt, i32([2, 2]), i32([3, 3]), res)
+    assert ctx.status() & b.ST_STATE
+    assert st.len_draft.tolist() == [0, 0] and ctx.launch_count() > n0
+    # a block-table entry outside the pool: BOUNDS bit, no fault
+    st.block_table[1, 0] = 1000
+    ctx.draft(st, i32([5, 6]))
+    assert ctx.status() & b.ST_BOUNDS
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    ctx.close()
