@@ -208,6 +208,9 @@ int64_t hispec_launch_count(const hispec_ctx *ctx);
 int hispec_profile_enable(hispec_ctx *ctx, int on);
 int hispec_profile_read(hispec_ctx *ctx, void *stream, int kind, double *ms, double *bytes, int64_t *launches);
 
+/* Text of the most recent CUDA failure behind a HISPEC_ECUDA return (process-wide, not thread-safe). */
+const char *hispec_last_error(void);
+
 /* Static text for an error code. */
 const char *hispec_strerror(int code);
 

@@ -25,7 +25,7 @@ ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["hispec_create", "hispec_destroy", "hispec_draft", "hispec_verify_intermediate", "hispec_verify_target",
            "hispec_prefill", "hispec_device_status", "hispec_launch_count", "hispec_strerror",
-           "hispec_profile_enable", "hispec_profile_read"]
+           "hispec_profile_enable", "hispec_profile_read", "hispec_last_error"]
 
 
 class ModelDesc(ctypes.Structure):
@@ -90,7 +90,8 @@ def load() -> ctypes.CDLL:
         lib.hispec_profile_enable.argtypes = [vp, i32]
         lib.hispec_profile_read.argtypes = [vp, vp, i32, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
-        for name in EXPORTS[:7] + EXPORTS[9:]:
+        lib.hispec_last_error.restype = ctypes.c_char_p
+        for name in EXPORTS[:7] + EXPORTS[9:11]:
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -102,7 +103,8 @@ class HiSpecError(RuntimeError):
 
 def _check(rc: int, what: str):
     if rc != 0:
-        raise HiSpecError(f"{what}: {load().hispec_strerror(rc).decode()} ({rc})")
+        detail = load().hispec_last_error().decode() if rc == -3 else ""
+        raise HiSpecError(f"{what}: {load().hispec_strerror(rc).decode()} ({rc}) {detail}")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:

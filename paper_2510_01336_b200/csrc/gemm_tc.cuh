@@ -21,6 +21,7 @@ namespace hispec {
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2..5: epilogue
 constexpr int kWTileBytes = kWeightTileRows * kTileK * 2;  // 16 KiB
+constexpr int kGemmMaxDynSmem = 220 * 1024;                // dynamic shared memory the kernel may be given
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {

@@ -146,10 +146,19 @@ struct ProfScope {
     }
 };
 
+static char g_last_error[256] = "";
+static void note_error(const char *what, int line, cudaError_t e) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s (line %d): %s", what, line, cudaGetErrorString(e));
+}
+extern "C" const char *hispec_last_error(void) { return g_last_error; }
+
 #define CK(expr)                              \
     do {                                      \
         cudaError_t e_ = (expr);              \
-        if (e_ != cudaSuccess) return HISPEC_ECUDA; \
+        if (e_ != cudaSuccess) {              \
+            note_error(#expr, __LINE__, e_);  \
+            return HISPEC_ECUDA;              \
+        }                                     \
     } while (0)
 
 extern "C" const char *hispec_strerror(int code) {
@@ -205,7 +214,11 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
             ok = ok && encode_2d(&c->tm_wdown[l], c->wdown[l], d.d_ffn, d.d_model, kWeightTileRows);
         }
     }
-    if (!ok) { hispec_destroy(c); return HISPEC_ECUDA; }
+    if (!ok) {
+        snprintf(g_last_error, sizeof(g_last_error), "cuTensorMapEncodeTiled failed for a weight matrix");
+        hispec_destroy(c);
+        return HISPEC_ECUDA;
+    }
 
     // split-K plan: enough CTAs to put every SM to work on each projection
     const int target = env_int("HISPEC_SPLIT_TARGET", c->sm_count);
@@ -255,17 +268,23 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     ok = ok && alloc((void **)&c->status, sizeof(uint32_t));
     if (!ok) { hispec_destroy(c); return HISPEC_ENOMEM; }
     bool e = true;
-    e = e && cudaMemset(c->status, 0, sizeof(uint32_t)) == cudaSuccess;
-    e = e && cudaMemset(c->act_d, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_model) == cudaSuccess;
-    e = e && cudaMemset(c->act_o, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * nq) == cudaSuccess;
-    e = e && cudaMemset(c->act_f, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_ffn) == cudaSuccess;
+    auto ck = [&](cudaError_t err, const char *what, int line) {
+        if (err != cudaSuccess && e) note_error(what, line, err);
+        e = e && err == cudaSuccess;
+    };
+#define CKB(expr) ck((expr), #expr, __LINE__)
+    CKB(cudaMemset(c->status, 0, sizeof(uint32_t)));
+    CKB(cudaMemset(c->act_d, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_model));
+    CKB(cudaMemset(c->act_o, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * nq));
+    CKB(cudaMemset(c->act_f, 0, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_ffn));
     // rotary frequencies base^(-2i/hd) in double precision
     int half = d.head_dim / 2;
     double *f = new double[half];
     for (int i = 0; i < half; ++i) f[i] = pow((double)d.rope_base, -2.0 * (double)i / (double)d.head_dim);
-    e = e && cudaMemcpy(c->inv_freq, f, sizeof(double) * half, cudaMemcpyHostToDevice) == cudaSuccess;
+    CKB(cudaMemcpy(c->inv_freq, f, sizeof(double) * half, cudaMemcpyHostToDevice));
     delete[] f;
-    e = e && cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+    CKB(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
+#undef CKB
     if (!e) { hispec_destroy(c); return HISPEC_ECUDA; }
     *out = c;
     return HISPEC_OK;
@@ -407,6 +426,7 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
         int stages = x->gemm_smem_budget / stage_bytes;
         if (stages < 2) stages = 2;
         if (stages > 16) stages = 16;
+        while (stages > 2 && (size_t)stages * stage_bytes + 1024 > (size_t)kGemmMaxDynSmem) --stages;
         g.stages = stages;
         g.head = head ? 1 : 0;
         g.part = c->part; g.split_stride = split_stride;

@@ -93,11 +93,12 @@ def compare_exit(out, res: binding.Result, b: int, n_rows: int, S, *, check_acce
 
 def compare_kv(st: binding.KVState, b: int, ost, page_size: int, layers, positions, tag: str = ""):
     """K/V appended by the call at `positions`: equal to the oracle's bf16-rounded entries up to one
-    bf16 rounding step (the two sides round nearly equal fp32 values independently)."""
+    bf16 rounding step (the two sides round nearly equal fp32 values independently) plus 2 % of the
+    entry's row RMS (bf16-rounded activations perturb small entries by more than their own ulp)."""
     bt = st.block_table[b].cpu()
     for l in layers:
         for pages, ref in ((st.k_pages, ost.cache.k), (st.v_pages, ost.cache.v)):
             g = cache_from_pages(pages, bt, page_size, l, st.first_layer, positions)
             r = ref[l, list(positions)]
-            tol = np.abs(r) * 2.0 ** -7 + 1e-3
+            tol = np.abs(r) * 2.0 ** -7 + 2e-2 * np.sqrt(np.mean(r.astype(np.float64) ** 2, axis=-1, keepdims=True))
             assert np.all(np.abs(g - r) <= tol), f"{tag} layer {l}: appended K/V differ"
