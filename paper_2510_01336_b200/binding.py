@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(HERE, "libhispec.so")
 FLAG_SIMT_GEMM = 1
 FLAG_PLAIN_ACT = 2
 FLAG_NO_PDL = 4
+FLAG_ROWWARP_ATTN = 8
 
 ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 

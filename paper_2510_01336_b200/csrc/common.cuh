@@ -60,6 +60,7 @@ struct hispec_ctx {
     size_t part_floats;
     float *attn_part;     // [T_max][hq][splits][hd + 2]
     int attn_max_splits;
+    size_t attn_part_floats;
     float *top_part;      // [vocab tiles][T_max][4]: v1, id1, v2, pad
     float *logits_ws;     // [kMaxGemmRows][vocab], SIMT debug path only
     double *inv_freq;     // [hd/2] rotary frequencies

@@ -69,6 +69,15 @@ int env_int(const char *name, int dflt) {
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
 
+// key splits of the tiled attention kernel: about four CTAs per SM over (batch, KV head, row group)
+inline int attn_splits(int sm_count, int batch, int hkv, int G, int R_pad) {
+    int n_mg = ceil_div(G * R_pad, 64);
+    int s = ceil_div(4 * sm_count, batch * hkv * n_mg);
+    if (s < 1) s = 1;
+    if (s > 64) s = 64;
+    return s;
+}
+
 struct ActMapCache {
     const void *base;
     int t_box, planes;
@@ -87,6 +96,8 @@ struct hispec_ctx_ext {
     bool profiling;
     std::vector<ProfEvent> *prof;       // recorded since the last read
     std::vector<ProfEvent> *prof_free;  // event pairs ready for reuse
+    struct PageMaps { const void *k, *v; long long n_pages; int pool_layers; CUtensorMap tmK, tmV; } page_maps[4];
+    int n_page_maps;
     ActMapCache act_cache[3][8];
     int act_cache_n[3];
     int T_alloc;
@@ -146,7 +157,7 @@ struct ProfScope {
     }
 };
 
-static char g_last_error[256] = "";
+static char g_last_error[640] = "";
 static void note_error(const char *what, int line, cudaError_t e) {
     snprintf(g_last_error, sizeof(g_last_error), "%s (line %d): %s", what, line, cudaGetErrorString(e));
 }
@@ -248,7 +259,17 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
         if (f > part_floats) part_floats = f;
     }
     c->part_floats = part_floats;
-    c->attn_max_splits = 1;
+    // split records of the tiled attention kernel: enough for the largest (batch, splits) product
+    {
+        size_t worst = 0;
+        for (int b = 1; b <= d.max_batch; ++b)
+            for (int r = 1; r <= d.max_rows_per_seq; ++r) {
+                size_t v = (size_t)attn_splits(c->sm_count, b, d.n_kv_heads, d.n_q_heads / d.n_kv_heads, r) * b * r;
+                if (v > worst) worst = v;
+            }
+        c->attn_max_splits = (int)(worst / ((size_t)d.max_batch * d.max_rows_per_seq)) + 1;
+        c->attn_part_floats = worst * d.n_q_heads * (d.head_dim + 2);
+    }
     auto alloc = [&](void **p, size_t bytes) { return cudaMalloc(p, bytes ? bytes : 16) == cudaSuccess; };
     ok = true;
     ok = ok && alloc((void **)&c->x, sizeof(float) * T_alloc * d.d_model);
@@ -257,6 +278,7 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     ok = ok && alloc((void **)&c->act_f, 2 * sizeof(__nv_bfloat16) * (size_t)T_alloc * d.d_ffn);
     ok = ok && alloc((void **)&c->q, sizeof(float) * (size_t)T_alloc * nq);
     ok = ok && alloc((void **)&c->part, sizeof(float) * part_floats);
+    ok = ok && alloc((void **)&c->attn_part, sizeof(float) * c->attn_part_floats);
     ok = ok && alloc((void **)&c->top_part, sizeof(float) * 4 * (size_t)c->plan[G_HEAD].tiles * 4 * T_alloc);
     if (simt) ok = ok && alloc((void **)&c->logits_ws, sizeof(float) * (size_t)T_alloc * d.vocab);
     ok = ok && alloc((void **)&c->inv_freq, sizeof(double) * (d.head_dim / 2));
@@ -293,7 +315,7 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
 extern "C" int hispec_destroy(hispec_ctx *c0) {
     if (!c0) return HISPEC_EINVAL;
     hispec_ctx_full *c = static_cast<hispec_ctx_full *>(c0);
-    void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->top_part, c->logits_ws, c->inv_freq,
+    void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->attn_part, c->top_part, c->logits_ws, c->inv_freq,
                     c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status};
     for (void *p : bufs)
         if (p) cudaFree(p);
@@ -322,7 +344,8 @@ extern "C" int hispec_profile_read(hispec_ctx *c, void *stream, int kind, double
     int64_t n = 0;
     std::vector<ProfEvent> keep;
     for (ProfEvent &e : *x->prof) {
-        if (e.kind != kind) { keep.push_back(e); continue; }
+        bool match = (kind == 0) ? (e.kind >= 10) : (e.kind == kind);
+        if (!match) { keep.push_back(e); continue; }
         float f = 0.0f;
         if (cudaEventElapsedTime(&f, e.a, e.b) == cudaSuccess) { t += f; by += e.bytes; ++n; }
         x->prof_free->push_back(e);
@@ -358,6 +381,26 @@ const CUtensorMap *act_map(hispec_ctx *c, int which, const void *base, int K, in
     if (!encode_act(&m.map, base, K, x->T_alloc, t_box, planes)) return nullptr;
     m.base = base; m.t_box = t_box; m.planes = planes;
     return &m.map;
+}
+
+// TMA descriptors over the caller's K and V page pools: rows = (layer, page, kv head, slot), box = one
+// page of one KV head, 64 dims wide
+const hispec_ctx_ext::PageMaps *page_maps(hispec_ctx *c, const hispec_kv &kv) {
+    hispec_ctx_ext *x = ext_of(c);
+    for (int i = 0; i < x->n_page_maps; ++i) {
+        auto &m = x->page_maps[i];
+        if (m.k == kv.k_pages && m.v == kv.v_pages && m.n_pages == kv.n_pages && m.pool_layers == kv.n_pool_layers)
+            return &m;
+    }
+    int slot = x->n_page_maps < 4 ? x->n_page_maps++ : 3;
+    auto &m = x->page_maps[slot];
+    uint64_t rows = (uint64_t)kv.n_pool_layers * kv.n_pages * c->d.n_kv_heads * c->d.page_size;
+    if (!encode_2d(&m.tmK, kv.k_pages, c->d.head_dim, rows, 16) || !encode_2d(&m.tmV, kv.v_pages, c->d.head_dim, rows, 16)) {
+        x->n_page_maps = slot;
+        return nullptr;
+    }
+    m.k = kv.k_pages; m.v = kv.v_pages; m.n_pages = kv.n_pages; m.pool_layers = kv.n_pool_layers;
+    return &m;
 }
 
 const CUtensorMap *head_map(hispec_ctx *c, const void *head) {
@@ -397,7 +440,7 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
     const int chunk = planes == 2 ? 128 : 256;
     for (int row0 = 0; row0 < T_pad; row0 += chunk) {
         int rows = T_pad - row0 < chunk ? T_pad - row0 : chunk;
-        ProfScope prof(c, st, 0, 2.0 * (double)p.N * (double)p.K);
+        ProfScope prof(c, st, 10 + (int)kind, 2.0 * (double)p.N * (double)p.K);
         if (simt) {
             float *outp = head ? c->logits_ws : c->part;
             dim3 grid(ceil_div(p.N * 32, 256), head ? 1 : p.splits);
@@ -481,12 +524,38 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         at.hq = d.n_q_heads; at.hkv = d.n_kv_heads; at.hd = d.head_dim;
         at.scale = 1.0f / sqrtf((float)d.head_dim);
         at.out = c->act_o; at.T_alloc = x->T_alloc; at.plain = plain;
-        {
+        const bool tiled = d.page_size == 16 && !(d.flags & HISPEC_FLAG_ROWWARP_ATTN);
+        if (!tiled) {
             ProfScope prof(c, st, 1, 0.0);
             int warps = T_pad * d.n_q_heads;
             dim3 grid(ceil_div(warps, 4));
             if (d.head_dim == 64) CK(launch(c, st, attention_rowwarp_kernel<64>, grid, dim3(128), 0, a, c->rows, at, c->status));
             else CK(launch(c, st, attention_rowwarp_kernel<128>, grid, dim3(128), 0, a, c->rows, at, c->status));
+        } else {
+            ProfScope prof(c, st, 1, 0.0);
+            const hispec_ctx_ext::PageMaps *pm = page_maps(c, kv);
+            if (!pm) return HISPEC_ECUDA;
+            AttnTcArgs ta;
+            ta.q = c->q; ta.block_table = kv.block_table; ta.n_pages = kv.n_pages; ta.pool_layer = pool_layer;
+            ta.hq = d.n_q_heads; ta.hkv = d.n_kv_heads; ta.G = d.n_q_heads / d.n_kv_heads;
+            const int QR = ta.G * a.R_pad;
+            ta.n_mg = ceil_div(QR, 64);
+            ta.mt = ceil_div(QR < 64 ? QR : 64, 16);
+            ta.n_splits = attn_splits(c->sm_count, a.batch, d.n_kv_heads, ta.G, a.R_pad);
+            ta.scale_log2 = at.scale * 1.4426950408889634f;
+            ta.part = c->attn_part;
+            if ((size_t)ta.n_splits * T_pad * d.n_q_heads * (d.head_dim + 2) > c->attn_part_floats) return HISPEC_ECAPACITY;
+            dim3 grid(ta.n_splits, d.n_kv_heads * ta.n_mg, a.batch), block((ta.mt + 1) * 32);
+            int mwarps = T_pad * d.n_q_heads;
+            if (d.head_dim == 64) {
+                CK(launch(c, st, attention_tc_kernel<64>, grid, block, 0, pm->tmK, pm->tmV, a, c->rows, ta, c->status));
+                CK(launch(c, st, attention_merge_kernel<64>, dim3(ceil_div(mwarps, 4)), dim3(128), 0, a, c->rows,
+                          (const float *)c->attn_part, ta.n_splits, d.n_q_heads, c->act_o, x->T_alloc, plain));
+            } else {
+                CK(launch(c, st, attention_tc_kernel<128>, grid, block, 0, pm->tmK, pm->tmV, a, c->rows, ta, c->status));
+                CK(launch(c, st, attention_merge_kernel<128>, dim3(ceil_div(mwarps, 4)), dim3(128), 0, a, c->rows,
+                          (const float *)c->attn_part, ta.n_splits, d.n_q_heads, c->act_o, x->T_alloc, plain));
+            }
         }
         if ((rc = run_gemm(c, st, G_O, c->wo[l], &c->tm_wo[l], 1, T_pad, sc)) != 0) return rc;
         CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, po.splits,
