@@ -210,6 +210,31 @@ int64_t hispec_launch_count(const hispec_ctx *ctx);
 int hispec_profile_enable(hispec_ctx *ctx, int on);
 int hispec_profile_read(hispec_ctx *ctx, void *stream, int kind, double *ms, double *bytes, int64_t *launches);
 
+/*
+ * Exit head + greedy token without any allocation (the paper has no counterpart; this is a
+ * service entry point for callers that cannot allocate device memory: a process whose free HBM was
+ * all given to its KV-page pool, a thread running while the allocator is held elsewhere, a plug-in
+ * that only receives raw pointers and a stream).  No hispec context is needed.
+ * For each of the n_rows hidden rows: z = head . RMSNorm(hidden[t]; final_norm); argmax_ids[t] = greedy
+ * token (lowest id on an exact tie), top2[t] = {largest, second largest logit} (top2 may be NULL).
+ *   head device bf16 [vocab][d_model]; final_norm device fp32 [d_model]; hidden device fp32
+ *   [n_rows][d_model]; argmax_ids device int32 [n_rows]; top2 device fp32 [n_rows][2].
+ * Limits: n_rows <= HISPEC_NOALLOC_MAX_ROWS, d_model <= HISPEC_NOALLOC_MAX_D, vocab <=
+ * HISPEC_NOALLOC_MAX_VOCAB; anything larger returns HISPEC_ECAPACITY and enqueues nothing.
+ * Scratch is a 1 MiB array compiled into the library, resident on every GPU that loads it, shared by
+ * all calls: calls whose kernels overlap on the GPU race with each other -- order them on one stream
+ * or with events.  The array keeps the previous call's contents; every element a call reads it has
+ * written first.  The first call on a device looks the array's address up
+ * (cudaGetSymbolAddress); make that first call outside stream capture.  Asynchronous on `stream`.
+ * The call uses no cudaMalloc / cudaFree and no allocating library routine.
+ */
+#define HISPEC_NOALLOC_MAX_ROWS 16
+#define HISPEC_NOALLOC_MAX_D 8192
+#define HISPEC_NOALLOC_MAX_VOCAB 262144
+int hispec_exit_argmax_noalloc(void *stream, const void *head, const float *final_norm, float rms_eps,
+                               int d_model, int vocab, const float *hidden, int n_rows, int32_t *argmax_ids,
+                               float *top2);
+
 /* Text of the most recent CUDA failure behind a HISPEC_ECUDA return (process-wide, not thread-safe). */
 const char *hispec_last_error(void);
 

@@ -26,7 +26,7 @@ ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["hispec_create", "hispec_destroy", "hispec_draft", "hispec_verify_intermediate", "hispec_verify_target",
            "hispec_prefill", "hispec_device_status", "hispec_launch_count", "hispec_strerror",
-           "hispec_profile_enable", "hispec_profile_read", "hispec_last_error"]
+           "hispec_profile_enable", "hispec_profile_read", "hispec_last_error", "hispec_exit_argmax_noalloc"]
 
 
 class ModelDesc(ctypes.Structure):
@@ -92,6 +92,8 @@ def load() -> ctypes.CDLL:
         lib.hispec_profile_read.argtypes = [vp, vp, i32, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
         lib.hispec_last_error.restype = ctypes.c_char_p
+        lib.hispec_exit_argmax_noalloc.argtypes = [vp, vp, vp, ctypes.c_float, i32, i32, vp, i32, vp, vp]
+        lib.hispec_exit_argmax_noalloc.restype = ctypes.c_int
         for name in EXPORTS[:7] + EXPORTS[9:11]:
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
@@ -289,3 +291,14 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.hispec_launch_count(self.handle))
+
+
+def exit_argmax_noalloc(head: torch.Tensor, final_norm: torch.Tensor, rms_eps: float, hidden: torch.Tensor,
+                        argmax_ids: torch.Tensor, top2: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Exit head + greedy token for hidden [n_rows][d] through the allocation-free entry point.
+    Outputs are written into the caller's tensors; nothing is allocated here or in the library."""
+    n_rows, d = hidden.shape
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _check(load().hispec_exit_argmax_noalloc(st.cuda_stream, _ptr(head), _ptr(final_norm), float(rms_eps), d,
+                                             head.shape[0], _ptr(hidden), n_rows, _ptr(argmax_ids), _ptr(top2)),
+           "hispec_exit_argmax_noalloc")

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhispec.so")
-SOURCES = ["hispec.cu"]
+SOURCES = ["hispec.cu", "noalloc.cu"]
 HEADERS = ["common.cuh", "kernels.cuh", "attention.cuh", "gemm_tc.cuh", os.path.join("..", "..", "include", "hispec.h")]
 
 
