@@ -53,6 +53,8 @@ extern "C" {
 #define HISPEC_FLAG_PLAIN_ACT 2u  /* feed bf16-rounded activations to the tensor cores (default: hi+lo split,
                                      x = bf16(x) + bf16(x - bf16(x)), which costs no extra HBM traffic) */
 #define HISPEC_FLAG_NO_PDL 4u     /* debug: launch kernels without programmatic dependent launch */
+#define HISPEC_FLAG_MULTI_KERNEL 16u /* run a call as a sequence of kernels instead of the single persistent kernel
+                                       (also taken when a call has more than 128 padded rows) */
 #define HISPEC_FLAG_ROWWARP_ATTN 8u /* debug: one-warp-per-row attention instead of the tiled kernel (the tiled
                                        kernel needs page_size == 16; other page sizes always take this path) */
 
@@ -201,7 +203,8 @@ int64_t hispec_launch_count(const hispec_ctx *ctx);
 
 /*
  * Measurement aid.  While profiling is enabled every projection (kind 0 = all projections; kinds
- * 10..14 = QKV, O, gate/up, down, exit head separately) and attention (kind 1) launch is bracketed by a pair of CUDA events on the call's stream, which also keeps neighbouring
+ * 10..14 = QKV, O, gate/up, down, exit head separately), attention (kind 1) and persistent whole-call
+ * (kind 20; bytes = weights of the layer range + exit head) launch is bracketed by a pair of CUDA events on the call's stream, which also keeps neighbouring
  * launches from overlapping.  hispec_profile_read() synchronises `stream`, adds up the event times
  * recorded since the last read into *ms, the weight bytes those projections streamed into *bytes
  * (0 for attention: the library does not know the context lengths on the host) and their number

@@ -21,6 +21,7 @@ FLAG_SIMT_GEMM = 1
 FLAG_PLAIN_ACT = 2
 FLAG_NO_PDL = 4
 FLAG_ROWWARP_ATTN = 8
+FLAG_MULTI_KERNEL = 16
 
 ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 

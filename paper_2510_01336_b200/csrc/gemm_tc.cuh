@@ -39,6 +39,25 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// bounded busy-poll variant (no hardware suspension between polls)
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
+    for (uint32_t it = 0; it < (1u << 28); ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((it & 65535u) == 65535u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicOr(status, HISPEC_ST_TIMEOUT);
+    return false;
+}
 // bounded wait; returns false (and raises the abort flag) when it gives up
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
     for (uint32_t it = 0; it < kSpinLimit; ++it) {

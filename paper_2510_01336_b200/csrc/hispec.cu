@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
+#include "mega.cuh"
 
 using namespace hispec;
 
@@ -93,6 +94,17 @@ struct ProfEvent {
 };
 
 struct hispec_ctx_ext {
+    // persistent-kernel path
+    bool mega_ok;              // cooperative launch available and the kernel fits
+    MegaGemm *d_gemms;         // device [n_layers * 4 + 4]: per-layer projections, then cached exit heads
+    const void *mega_heads[4];
+    int n_mega_heads;
+    const float **d_attn_norm, **d_ffn_norm;  // device arrays of device pointers
+    float *ssq;                // [T_alloc][ceil(d / 256)] chunk sums of squares
+    unsigned *bar;             // grid barrier counters, used alternately by successive launches
+    int bar_sel;
+    unsigned long long *trace; // debug: phase time stamps of the persistent kernel (HISPEC_TRACE=1)
+    size_t mega_part_floats[4];  // partial-sum floats per padded row the stream-K partition needs, per projection
     bool profiling;
     std::vector<ProfEvent> *prof;       // recorded since the last read
     std::vector<ProfEvent> *prof_free;  // event pairs ready for reuse
@@ -258,6 +270,24 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
         size_t f = (size_t)c->plan[k].splits * T_alloc * c->plan[k].N;
         if (f > part_floats) part_floats = f;
     }
+    // persistent-kernel path: stream-K partial slots per tile (one per CTA whose span touches the tile)
+    {
+        const int G = c->sm_count;
+        for (int k = 0; k < G_HEAD; ++k) {
+            const GemmPlan &p = c->plan[k];
+            const long long U = (long long)p.tiles * p.kb_total;
+            int smax = 1;
+            (void)U;
+            for (int tile = 0; tile < p.tiles; ++tile) {
+                int first, ns;
+                mega_slots(tile, p.tiles, p.kb_total, G, first, ns);
+                if (ns > smax) smax = ns;
+            }
+            c->ext.mega_part_floats[k] = (size_t)smax * p.N;
+            size_t f = (size_t)smax * T_alloc * p.N;
+            if (f > part_floats) part_floats = f;
+        }
+    }
     c->part_floats = part_floats;
     // split records of the tiled attention kernel: enough for the largest (batch, splits) product
     {
@@ -288,6 +318,12 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     ok = ok && alloc((void **)&c->rows.dst_row, sizeof(int32_t) * d.max_batch);
     ok = ok && alloc((void **)&c->argmax_ws, sizeof(int32_t) * T_alloc);
     ok = ok && alloc((void **)&c->status, sizeof(uint32_t));
+    ok = ok && alloc((void **)&c->ext.d_gemms, sizeof(MegaGemm) * (L * 4 + 4));
+    ok = ok && alloc((void **)&c->ext.d_attn_norm, sizeof(float *) * L);
+    ok = ok && alloc((void **)&c->ext.d_ffn_norm, sizeof(float *) * L);
+    ok = ok && alloc((void **)&c->ext.ssq, sizeof(float) * (size_t)T_alloc * ceil_div(d.d_model, kEwChunk));
+    ok = ok && alloc((void **)&c->ext.bar, 2 * sizeof(unsigned));
+    if (env_int("HISPEC_TRACE", 0)) ok = ok && alloc((void **)&c->ext.trace, 1024 * sizeof(unsigned long long));
     if (!ok) { hispec_destroy(c); return HISPEC_ENOMEM; }
     bool e = true;
     auto ck = [&](cudaError_t err, const char *what, int line) {
@@ -306,6 +342,29 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     CKB(cudaMemcpy(c->inv_freq, f, sizeof(double) * half, cudaMemcpyHostToDevice));
     delete[] f;
     CKB(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
+    CKB(cudaMemset(c->ext.bar, 0, 2 * sizeof(unsigned)));
+    CKB(cudaMemcpy(c->ext.d_attn_norm, c->attn_norm, sizeof(float *) * L, cudaMemcpyHostToDevice));
+    CKB(cudaMemcpy(c->ext.d_ffn_norm, c->ffn_norm, sizeof(float *) * L, cudaMemcpyHostToDevice));
+    if (!simt) {
+        // device table of projection descriptors for the persistent kernel
+        std::vector<MegaGemm> hg((size_t)L * 4 + 4);
+        memset(hg.data(), 0, sizeof(MegaGemm) * hg.size());
+        for (int l = 0; l < L; ++l) {
+            const CUtensorMap *tms[4] = {&c->tm_wqkv[l], &c->tm_wo[l], &c->tm_wgu[l], &c->tm_wdown[l]};
+            for (int k = 0; k < 4; ++k) {
+                MegaGemm &g = hg[(size_t)l * 4 + k];
+                if (c->wqkv[l]) g.tmW = *tms[k];
+                g.N = c->plan[k].N; g.K = c->plan[k].K; g.tiles = c->plan[k].tiles; g.kb_total = c->plan[k].kb_total;
+            }
+        }
+        CKB(cudaMemcpy(c->ext.d_gemms, hg.data(), sizeof(MegaGemm) * hg.size(), cudaMemcpyHostToDevice));
+        CKB(cudaFuncSetAttribute(hispec_stage_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
+        CKB(cudaFuncSetAttribute(hispec_stage_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
+        int coop = 0;
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
+        c->ext.mega_ok = coop != 0 && d.page_size == 16 && d.max_batch <= kMegaMaxBatch &&
+                         !(d.flags & (HISPEC_FLAG_MULTI_KERNEL | HISPEC_FLAG_ROWWARP_ATTN));
+    }
 #undef CKB
     if (!e) { hispec_destroy(c); return HISPEC_ECUDA; }
     *out = c;
@@ -316,7 +375,8 @@ extern "C" int hispec_destroy(hispec_ctx *c0) {
     if (!c0) return HISPEC_EINVAL;
     hispec_ctx_full *c = static_cast<hispec_ctx_full *>(c0);
     void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->attn_part, c->top_part, c->logits_ws, c->inv_freq,
-                    c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status};
+                    c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status,
+                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace};
     for (void *p : bufs)
         if (p) cudaFree(p);
     delete[] c->wqkv; delete[] c->wo; delete[] c->wgu; delete[] c->wdown; delete[] c->attn_norm; delete[] c->ffn_norm;
@@ -344,7 +404,7 @@ extern "C" int hispec_profile_read(hispec_ctx *c, void *stream, int kind, double
     int64_t n = 0;
     std::vector<ProfEvent> keep;
     for (ProfEvent &e : *x->prof) {
-        bool match = (kind == 0) ? (e.kind >= 10) : (e.kind == kind);
+        bool match = (kind == 0) ? (e.kind >= 10 && e.kind < 20) : (e.kind == kind);
         if (!match) { keep.push_back(e); continue; }
         float f = 0.0f;
         if (cudaEventElapsedTime(&f, e.a, e.b) == cudaSuccess) { t += f; by += e.bytes; ++n; }
@@ -353,6 +413,15 @@ extern "C" int hispec_profile_read(hispec_ctx *c, void *stream, int kind, double
     x->prof->swap(keep);
     *ms = t; *bytes = by; *launches = n;
     return HISPEC_OK;
+}
+
+// debug: copy the persistent kernel's phase time stamps (ns) of the last call; returns their number
+extern "C" int hispec_debug_trace(hispec_ctx *c, unsigned long long *out, int cap) {
+    hispec_ctx_ext *x = ext_of(c);
+    if (!x->trace || cap < 1024) return 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return 0;
+    if (cudaMemcpy(out, x->trace, 1024 * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) return 0;
+    return 1024;
 }
 
 extern "C" int64_t hispec_launch_count(const hispec_ctx *c) { return c ? c->launches : 0; }
@@ -364,6 +433,10 @@ extern "C" int hispec_device_status(hispec_ctx *c, void *stream, uint32_t *host_
     CK(cudaMemcpyAsync(host_out, c->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaMemsetAsync(c->status, 0, sizeof(uint32_t), st));
     CK(cudaStreamSynchronize(st));
+    if (*host_out & HISPEC_ST_TIMEOUT) {  // a kernel that gave up may have left the grid barrier half way
+        CK(cudaMemset(ext_of(c)->bar, 0, 2 * sizeof(unsigned)));
+        ext_of(c)->bar_sel = 0;
+    }
     return HISPEC_OK;
 }
 
@@ -485,7 +558,124 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
     return HISPEC_OK;
 }
 
+// index of the exit head's descriptor in the device table (encoded and uploaded on first use)
+int mega_head_slot(hispec_ctx *c, const void *head) {
+    hispec_ctx_ext *x = ext_of(c);
+    for (int i = 0; i < x->n_mega_heads; ++i)
+        if (x->mega_heads[i] == head) return i;
+    int slot = x->n_mega_heads < 4 ? x->n_mega_heads : 3;
+    MegaGemm g;
+    memset(&g, 0, sizeof(g));
+    if (!encode_2d(&g.tmW, head, c->d.d_model, c->d.vocab, kWeightTileRows)) return -1;
+    const GemmPlan &p = c->plan[G_HEAD];
+    g.N = p.N; g.K = p.K; g.tiles = p.tiles; g.kb_total = p.kb_total;
+    if (cudaMemcpy(x->d_gemms + (size_t)c->d.n_layers * 4 + slot, &g, sizeof(g), cudaMemcpyHostToDevice) != cudaSuccess)
+        return -1;
+    x->mega_heads[slot] = head;
+    if (x->n_mega_heads < 4) x->n_mega_heads++;
+    return slot;
+}
+
+// the whole call as one cooperative launch of the persistent kernel; returns 1 if the call does not fit it
+int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
+    const hispec_model_desc &d = c->d;
+    hispec_ctx_ext *x = ext_of(c);
+    const StageArgs &a = sc.a;
+    const int T_pad = a.batch * a.R_pad;
+    const int plain = (d.flags & HISPEC_FLAG_PLAIN_ACT) ? 1 : 0;
+    const int planes = plain ? 1 : 2;
+    if (!x->mega_ok || T_pad * planes > kMegaAccCols) return 1;
+    const hispec_kv &kv = *sc.kv;
+    MegaArgs m;
+    memset(&m, 0, sizeof(m));
+    m.a = a;
+    m.gemms = x->d_gemms;
+    const void *head = (a.l1 == a.L_d) ? sc.exits->head_d : ((a.l1 == a.L_i) ? sc.exits->head_i : sc.exits->head_f);
+    int hs = mega_head_slot(c, head);
+    if (hs < 0) return HISPEC_ECUDA;
+    m.head = x->d_gemms + (size_t)d.n_layers * 4 + hs;
+    m.attn_norm = x->d_attn_norm; m.ffn_norm = x->d_ffn_norm; m.final_norm = c->final_norm;
+    m.d = d.d_model; m.hq = d.n_q_heads; m.hkv = d.n_kv_heads; m.hd = d.head_dim; m.ffn = d.d_ffn; m.vocab = d.vocab;
+    m.eps = d.rms_eps;
+    m.T_pad = T_pad; m.T_alloc = x->T_alloc; m.planes = planes; m.plain = plain;
+    m.t_box = round_up(T_pad, planes == 2 ? 8 : 16);
+    const int ncols = m.t_box * planes;
+    const int attn_bytes = kAttnStages * 2 * 16 * d.head_dim * 2;
+    const int stage_bytes = kWTileBytes + ncols * 128;
+    int stages = (kGemmMaxDynSmem - attn_bytes - 1024) / (2 * stage_bytes);  // two pipelines
+    int cap = env_int("HISPEC_MEGA_STAGES", kMegaMaxStages);
+    if (stages > cap) stages = cap;
+    if (stages > kMegaMaxStages) stages = kMegaMaxStages;
+    if (stages < 2) return 1;
+    m.stages = stages;
+    for (int k = 0; k < G_HEAD; ++k)
+        if (x->mega_part_floats[k] * (size_t)T_pad > c->part_floats) return 1;
+    m.len_d = kv.len_draft; m.len_i = kv.len_inter; m.len_f = kv.len_target;
+    m.n_rows_in = sc.n_rows; m.n_draft_in = sc.n_draft; m.tokens = sc.tokens; m.n_tokens = sc.n_tokens;
+    m.tok_emb = (const __nv_bfloat16 *)c->tok_emb;
+    if (a.mode == 1) m.h_src = (a.l0 == a.L_d) ? sc.hidden->h_draft : sc.hidden->h_inter;
+    if (a.l1 == a.L_d) m.exit_buf = sc.hidden ? sc.hidden->h_draft : nullptr;
+    else if (a.l1 == a.L_i) m.exit_buf = sc.hidden ? sc.hidden->h_inter : nullptr;
+    m.hidden_out = sc.res ? sc.res->hidden_out : nullptr;
+    m.k_pages = (__nv_bfloat16 *)kv.k_pages; m.v_pages = (__nv_bfloat16 *)kv.v_pages;
+    m.block_table = kv.block_table; m.n_pages = kv.n_pages; m.first_layer = kv.first_layer;
+    m.x = c->x; m.act_d = c->act_d; m.act_o = c->act_o; m.act_f = c->act_f; m.q = c->q; m.part = c->part;
+    m.attn_part = c->attn_part; m.top_part = c->top_part; m.ssq = x->ssq; m.inv_freq = c->inv_freq;
+    m.G = d.n_q_heads / d.n_kv_heads;
+    const int QR = m.G * a.R_pad;
+    m.n_mg = ceil_div(QR, 64);
+    m.mt = ceil_div(QR < 64 ? QR : 64, 16);
+    // one attention item per CTA where possible: the phase is latency-bound at small batch
+    m.n_splits = c->sm_count / (a.batch * d.n_kv_heads * m.n_mg);
+    if (m.n_splits < 1) m.n_splits = 1;
+    if (m.n_splits > 64) m.n_splits = 64;
+    if ((size_t)m.n_splits * T_pad * d.n_q_heads * (d.head_dim + 2) > c->attn_part_floats) return 1;
+    m.scale_log2 = (1.0f / sqrtf((float)d.head_dim)) * 1.4426950408889634f;
+    m.r.len_d = kv.len_draft; m.r.len_i = kv.len_inter; m.r.len_f = kv.len_target;
+    m.r.draft_tokens = sc.draft_tokens; m.r.token_stride = sc.token_stride; m.r.out_stride = sc.out_stride;
+    if (sc.res) {
+        m.r.n_accepted = sc.res->n_accepted; m.r.next_token = sc.res->next_token;
+        m.r.argmax_ids = sc.res->argmax_ids; m.r.top2 = sc.res->top2; m.r.tentative = sc.res->tentative;
+        m.r.pending = sc.res->pending;
+        m.logits = sc.res->logits;
+    }
+    m.r.out_tokens = sc.out_tokens; m.r.n_tokens = sc.n_tokens;
+    m.argmax_ws = c->argmax_ws;
+    m.status = c->status;
+    m.bar_count = x->bar + (x->bar_sel & 1); m.bar_next = x->bar + ((x->bar_sel + 1) & 1);
+    x->bar_sel ^= 1;
+    m.trace = x->trace;
+    const CUtensorMap *tmd = act_map(c, 0, c->act_d, d.d_model, m.t_box, planes);
+    const CUtensorMap *tmo = act_map(c, 1, c->act_o, d.n_q_heads * d.head_dim, m.t_box, planes);
+    const CUtensorMap *tmf = act_map(c, 2, c->act_f, d.d_ffn, m.t_box, planes);
+    const hispec_ctx_ext::PageMaps *pm = page_maps(c, kv);
+    if (!tmd || !tmo || !tmf || !pm) return HISPEC_ECUDA;
+    const size_t smem = (size_t)2 * stages * stage_bytes + attn_bytes + 1024;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->sm_count);
+    cfg.blockDim = dim3(kMegaThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    c->launches++;
+    double wbytes = 2.0 * (double)c->plan[G_HEAD].N * c->plan[G_HEAD].K;
+    for (int k = 0; k < G_HEAD; ++k) wbytes += 2.0 * (double)c->plan[k].N * c->plan[k].K * (a.l1 - a.l0);
+    ProfScope prof(c, st, 20, wbytes);
+    if (d.head_dim == 64) CK(cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m));
+    else CK(cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m));
+    return HISPEC_OK;
+}
+
 int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
+    {
+        int rc = run_stage_mega(c, st, sc);
+        if (rc != 1) return rc;
+    }
     const hispec_model_desc &d = c->d;
     const StageArgs &a = sc.a;
     hispec_ctx_ext *x = ext_of(c);

@@ -1,0 +1,1070 @@
+// One persistent kernel per stage call: every step a0..a10 of the call runs inside a single
+// cooperative launch with one CTA per SM.
+//
+// Why: at batch 1 a call is ~80 dependent kernels of 5-50 us each, and every kernel boundary
+// drains the HBM pipe for several microseconds.  Here the weights -- which depend on nothing
+// the call computes -- are streamed by a dedicated TMA warp that runs through the *whole*
+// call's schedule of weight tiles, limited only by free slots in a deep shared-memory ring, so
+// HBM keeps flowing across the dependency points (grid barriers, attention, element-wise
+// phases).  The other warps work phase by phase:
+//
+//   projection phase   two independent pipelines per CTA (measured: one TMA ring + one MMA thread
+//                      per SM tops out near 4.9 TB/s, two reach the HBM limit): warps 0/1 stream
+//                      weights, warps 2/3 issue tcgen05.mma (accumulators in TMEM, double
+//                      buffered per pipeline), warps 4/5 TMA-load the activation operand, warps
+//                      6-9 drain TMEM to split-K partial sums (stream-K partition over 2 x grid
+//                      "virtual CTAs": every pipeline gets the same number of 128x64 weight
+//                      blocks, +-1), or, for the exit head, to top-2 records (there the two
+//                      pipelines take the two halves of each tile's K range);
+//   element-wise phase warps 2-9 of all CTAs: sum the partial slots in slot order, then
+//                      RoPE + KV append / residual + gain + hi-lo split / SiLU*up / split merge;
+//   attention phase    warp 5 stages KV pages by TMA, warps 6-9 run the tiled attention;
+//   final phase        CTA b reduces sequence b's top-2 records and applies LeadingSubstringVerify.
+//
+// RMSNorm is applied as y = W (g .* x) / rms(x): the projection runs on g .* x and the row's
+// 1/rms (from per-chunk sums of squares written by the producing phase) scales the result where
+// the partial sums are consumed, so no grid barrier is needed between "residual" and "norm".
+//
+// Phases are separated by a grid barrier (counter + generation word in global memory).  Every
+// wait -- mbarrier or grid barrier -- is bounded; on a timeout the CTA raises an abort flag,
+// sets HISPEC_ST_TIMEOUT, and all later waits fall through so that the kernel drains and exits.
+#pragma once
+
+#include "attention.cuh"
+#include "gemm_tc.cuh"
+
+namespace hispec {
+
+constexpr int kMegaThreads = 320;
+constexpr int kMegaMaxStages = 8;  // per pipeline
+constexpr int kMegaMaxBatch = 64;
+constexpr int kMegaWorkers = 256;  // threads of warps 2..9
+constexpr int kMegaLeader = 64;    // warp 2 lane 0
+constexpr int kMegaAccCols = 128;  // TMEM columns per accumulator buffer (2 pipelines x 2 buffers)
+constexpr int kEwChunk = 256;      // columns per element-wise work item (one warp, 8 per lane)
+
+struct __align__(64) MegaGemm {
+    CUtensorMap tmW;
+    int N, K, tiles, kb_total;
+    int pad[12];
+};
+
+struct MegaArgs {
+    StageArgs a;
+    const MegaGemm *gemms;  // [n_layers][4]: QKV, O, gate/up, down
+    const MegaGemm *head;
+    const float *const *attn_norm;
+    const float *const *ffn_norm;
+    const float *final_norm;
+    int d, hq, hkv, hd, ffn, vocab;
+    float eps;
+    int T_pad, T_alloc, t_box, planes, stages, plain;
+    int32_t *len_d, *len_i, *len_f;
+    const int32_t *n_rows_in, *n_draft_in, *tokens, *n_tokens;
+    const __nv_bfloat16 *tok_emb;
+    const float *h_src;
+    float *exit_buf, *hidden_out;
+    __nv_bfloat16 *k_pages, *v_pages;
+    const int32_t *block_table;
+    long long n_pages;
+    int first_layer;
+    float *x;
+    __nv_bfloat16 *act_d, *act_o, *act_f;
+    float *q, *part, *attn_part, *top_part, *ssq;
+    const double *inv_freq;
+    int n_splits, n_mg, mt, G;
+    float scale_log2;
+    AcceptArgs r;
+    int32_t *argmax_ws;
+    float *logits;
+    uint32_t *status;
+    unsigned *bar_count;     // this launch's barrier counter (zero at launch)
+    unsigned *bar_next;      // the next launch's counter: zeroed by this launch
+    unsigned long long *trace;  // optional: CTA 0 stamps the global timer after every grid barrier
+};
+
+struct MegaShared {
+    uint64_t w_full[2][kMegaMaxStages], x_full[2][kMegaMaxStages], empty[2][kMegaMaxStages];
+    uint64_t acc_full[2][2], acc_empty[2][2];
+    uint64_t a_full[kAttnStages], a_empty[kAttnStages];
+    uint32_t tmem;
+    int abort_flag;
+    int trace_n;
+    int bar_k;
+    int p0[kMegaMaxBatch], nr[kMegaMaxBatch], nd[kMegaMaxBatch], dst[kMegaMaxBatch];
+    float red_v1[8], red_v2[8];
+    int red_i1[8];
+};
+
+// ---- stream-K partition ----------------------------------------------------------------------
+// The k-blocks of a projection, numbered tile-major, are cut into gridDim.x equal spans.
+__host__ __device__ inline int mega_eff_ctas(long long U, int G) { return U < (long long)G ? (int)U : G; }
+__host__ __device__ inline int mega_cta_of(long long u, long long U, int G) {
+    return (int)(((u + 1) * G + U - 1) / U) - 1;
+}
+// Pipeline p of CTA c is virtual CTA 2c + p of 2G.  In `whole` mode (exit head: the epilogue needs a
+// tile's complete K range) tiles are dealt to real CTAs and pipeline p takes half p of each tile's K range.
+struct SegIter {
+    long long u, hi;
+    int kbt, whole, p;
+    __device__ SegIter(int tiles, int kb_total, int whole_, int c, int p_, int G) : kbt(kb_total), whole(whole_), p(p_) {
+        if (whole) {
+            u = (long long)c * tiles / G;        // tile index range
+            hi = (long long)(c + 1) * tiles / G;
+        } else {
+            long long U = (long long)tiles * kb_total;
+            int Ge = mega_eff_ctas(U, 2 * G);    // with fewer k-blocks than pipelines only the first U take part
+            int vc = 2 * c + p;
+            if (vc >= Ge) { u = hi = 0; return; }
+            u = (long long)vc * U / Ge;
+            hi = (long long)(vc + 1) * U / Ge;
+        }
+    }
+    __device__ bool next(int &tile, int &kb0, int &kb1) {
+        if (u >= hi) return false;
+        if (whole) {
+            tile = (int)u;
+            kb0 = p ? kbt / 2 : 0;
+            kb1 = p ? kbt : kbt / 2;
+            ++u;
+            return true;
+        }
+        tile = (int)(u / kbt);
+        kb0 = (int)(u % kbt);
+        long long rem = hi - u;
+        kb1 = (rem < (long long)(kbt - kb0)) ? kb0 + (int)rem : kbt;
+        u += kb1 - kb0;
+        return true;
+    }
+};
+// slots of a tile: one per CTA whose span touches it, in CTA order
+__host__ __device__ inline void mega_slots(int tile, int tiles, int kbt, int G, int &first_cta, int &n_slots) {
+    long long U = (long long)tiles * kbt;
+    int Ge = mega_eff_ctas(U, 2 * G);
+    first_cta = mega_cta_of((long long)tile * kbt, U, Ge);
+    n_slots = mega_cta_of((long long)(tile + 1) * kbt - 1, U, Ge) - first_cta + 1;
+}
+
+// ---- barriers --------------------------------------------------------------------------------
+__device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kMegaWorkers) : "memory"); }
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// All worker threads of all CTAs.  Global writes made before it are visible after it, also to TMA
+// reads.  The counter only grows during a launch: barrier number k is passed once it has reached
+// (k + 1) * gridDim.x.  Arrival is a fire-and-forget release reduction; waiting polls with acquire loads.
+__device__ __forceinline__ void grid_sync(const MegaArgs &m, MegaShared &sh) {
+    asm volatile("fence.proxy.async;" ::: "memory");
+    worker_bar();
+    if (threadIdx.x == kMegaLeader) {
+        volatile int *ab = &sh.abort_flag;
+        const unsigned target = (unsigned)(++sh.bar_k) * gridDim.x;
+        if (!*ab) {
+            asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(m.bar_count) : "memory");
+            bool ok = false;
+            for (uint32_t it = 0; it < (1u << 26); ++it) {
+                if ((int)(ld_acquire_u32(m.bar_count) - target) >= 0) { ok = true; break; }
+                if ((it & 4095u) == 4095u && (*((volatile uint32_t *)m.status) & HISPEC_ST_TIMEOUT)) break;
+            }
+            if (!ok) {
+                *ab = 1;
+                atomicOr(m.status, HISPEC_ST_TIMEOUT);
+            }
+        }
+        if (m.trace && blockIdx.x == 0) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+            int i = sh.trace_n++;
+            if (i < 1000) m.trace[i] = t;
+        }
+    }
+    worker_bar();
+}
+
+// ---- row bookkeeping (every CTA computes the same table; CTA 0 reports) -------------------------
+__device__ __forceinline__ void mega_prep_rows(const MegaArgs &m, MegaShared &sh) {
+    const StageArgs &a = m.a;
+    for (int b = threadIdx.x; b < a.batch; b += blockDim.x) {
+        int gA = m.len_d[b], gB = m.len_i[b], gC = m.len_f[b];
+        int p0 = a.l0 < a.L_d ? gA : (a.l0 < a.L_i ? gB : gC);
+        uint32_t st = 0;
+        int nr, nd = 0;
+        if (a.mode == 0) {
+            if (m.n_tokens) {
+                nr = m.n_tokens[b] - a.tok_offset;
+                nr = nr < 0 ? 0 : (nr > a.R_pad ? a.R_pad : nr);
+            } else {
+                nr = a.fixed_rows;
+                if (m.tokens[b * a.tok_stride + a.tok_offset] < 0) nr = 0;
+            }
+        } else if (m.n_rows_in) {
+            nr = m.n_rows_in[b];
+            nd = m.n_draft_in[b];
+            if (nr < 0 || nr > a.R_pad || nd < 0 || nd > nr || nr > nd + 1 || nd > a.k) { st |= HISPEC_ST_STATE; nr = 0; nd = 0; }
+        } else {
+            int avail = (a.l0 == a.L_d) ? gA - gB : gB - gC;
+            if (avail < 0) avail = 0;
+            if (a.is_target && avail > a.k) st |= HISPEC_ST_STATE;
+            nr = avail < a.R_pad ? avail : a.R_pad;
+            nd = nr < a.k ? nr : a.k;
+        }
+        if (a.l0 < a.L_d && a.l1 > a.L_d && gB != p0) st |= HISPEC_ST_STATE;
+        if (a.l0 < a.L_i && a.l1 > a.L_i && gC != p0) st |= HISPEC_ST_STATE;
+        if (gC > gB || gB > gA) st |= HISPEC_ST_STATE;
+        if (a.mode == 1) {
+            int avail = (a.l0 == a.L_d) ? gA - gB : gB - gC;
+            if (avail < nr) st |= HISPEC_ST_STATE;
+        }
+        int dst = (a.l1 == a.L_d) ? p0 - gB : ((a.l1 == a.L_i) ? p0 - gC : 0);
+        if (a.l1 != a.L_f && (dst < 0 || dst + nr > a.max_rows)) st |= HISPEC_ST_BOUNDS;
+        if ((long long)p0 + nr > (long long)a.max_pages * a.page_size || p0 < 0) st |= HISPEC_ST_BOUNDS;
+        if (st) {
+            if (blockIdx.x == 0) atomicOr(m.status, st);
+            nr = 0;
+            nd = 0;
+        }
+        sh.p0[b] = p0; sh.nr[b] = nr; sh.nd[b] = nd; sh.dst[b] = dst;
+    }
+}
+
+// 1 / rms of row t from the per-chunk sums of squares of the phase that produced the row
+__device__ __forceinline__ float mega_inv_rms(const MegaArgs &m, int t) {
+    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
+    float s = 0.f;
+    for (int c = 0; c < nch; ++c) s += m.ssq[(size_t)t * nch + c];
+    return rsqrtf(s / (float)m.d + m.eps);
+}
+
+__device__ __forceinline__ void store8_hilo(__nv_bfloat16 *hi, __nv_bfloat16 *lo, const float *v, int plain) {
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat16 h0, l0, h1, l1;
+        split_hi_lo(v[2 * i], h0, l0, plain);
+        split_hi_lo(v[2 * i + 1], h1, l1, plain);
+        __nv_bfloat162 hh = __halves2bfloat162(h0, h1), ll = __halves2bfloat162(l0, l1);
+        h[i] = *reinterpret_cast<uint32_t *>(&hh);
+        l[i] = *reinterpret_cast<uint32_t *>(&ll);
+    }
+    *reinterpret_cast<uint4 *>(hi) = make_uint4(h[0], h[1], h[2], h[3]);
+    *reinterpret_cast<uint4 *>(lo) = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+// sum of the split-K partial slots of 8 consecutive columns (all inside one tile), slot order
+__device__ __forceinline__ void sum_slots8(const MegaArgs &m, const MegaGemm &g, int t, int n, float *v) {
+    int first, ns;
+    mega_slots(n / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
+    const size_t stride = (size_t)m.T_pad * g.N;
+    const float *p = m.part + (size_t)t * g.N + n;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = 0.f;
+    for (int s = 0; s < ns; ++s) {
+        float4 a = *reinterpret_cast<const float4 *>(p + s * stride);
+        float4 b = *reinterpret_cast<const float4 *>(p + s * stride + 4);
+        v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+        v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+    }
+}
+__device__ __forceinline__ float sum_slots1(const MegaArgs &m, const MegaGemm &g, int t, int n) {
+    int first, ns;
+    mega_slots(n / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
+    const size_t stride = (size_t)m.T_pad * g.N;
+    const float *p = m.part + (size_t)t * g.N + n;
+    float v = 0.f;
+    for (int s = 0; s < ns; ++s) v += p[s * stride];
+    return v;
+}
+
+// ---- element-wise phases (gw: global worker-warp index, ngw: number of worker warps in the grid) ----
+// a0 + gain: fetch rows, x <- row, act_d <- hi/lo(x .* gain), chunk sums of squares
+__device__ void ew_rows_in(const MegaArgs &m, MegaShared &sh, const float *gain, int gw, int ngw, int lane) {
+    const StageArgs &a = m.a;
+    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
+    for (int item = gw; item < m.T_pad * nch; item += ngw) {
+        const int t = item / nch, ch = item % nch, b = t / a.R_pad, j = t % a.R_pad;
+        const int c = ch * kEwChunk + lane * 8;
+        bool valid = j < sh.nr[b];
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        if (valid && c < m.d) {
+            if (a.mode == 0) {
+                int tok = m.tokens[b * a.tok_stride + a.tok_offset + j];
+                if (tok < 0 || tok >= m.vocab) {
+                    if (lane == 0 && ch == 0) atomicOr(m.status, HISPEC_ST_BOUNDS);
+                } else {
+                    uint4 raw = *reinterpret_cast<const uint4 *>(m.tok_emb + (size_t)tok * m.d + c);
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        v[2 * i] = __uint_as_float(w[i] << 16);
+                        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+                    }
+                }
+            } else {
+                const float *src = m.h_src + ((size_t)b * a.max_rows + j) * m.d + c;
+                float4 p = *reinterpret_cast<const float4 *>(src), q = *reinterpret_cast<const float4 *>(src + 4);
+                v[0] = p.x; v[1] = p.y; v[2] = p.z; v[3] = p.w; v[4] = q.x; v[5] = q.y; v[6] = q.z; v[7] = q.w;
+            }
+        }
+        float ss = 0.f;
+        if (c < m.d) {
+            float *xr = m.x + (size_t)t * m.d + c;
+            *reinterpret_cast<float4 *>(xr) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4 *>(xr + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            float gv[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { ss += v[i] * v[i]; gv[i] = v[i] * gain[c + i]; }
+            store8_hilo(m.act_d + (size_t)t * m.d + c, m.act_d + ((size_t)m.T_alloc + t) * m.d + c, gv, m.plain);
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) m.ssq[(size_t)t * nch + ch] = ss;
+    }
+}
+
+// a5/a7 epilogue: x += projection; act_d <- hi/lo(x .* gain); chunk sums of squares; exit rows on the last layer
+__device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, const float *gain, float *exit_buf,
+                         float *hidden_out, int gw, int ngw, int lane) {
+    const StageArgs &a = m.a;
+    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
+    for (int item = gw; item < m.T_pad * nch; item += ngw) {
+        const int t = item / nch, ch = item % nch, b = t / a.R_pad, j = t % a.R_pad;
+        const int c = ch * kEwChunk + lane * 8;
+        const bool valid = j < sh.nr[b];
+        float ss = 0.f;
+        if (c < m.d) {
+            float v[8];
+            sum_slots8(m, g, t, c, v);
+            float *xr = m.x + (size_t)t * m.d + c;
+            float4 p = *reinterpret_cast<const float4 *>(xr), q = *reinterpret_cast<const float4 *>(xr + 4);
+            const float xo[8] = {p.x, p.y, p.z, p.w, q.x, q.y, q.z, q.w};
+            float gv[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[i] = valid ? v[i] + xo[i] : 0.f;
+                ss += v[i] * v[i];
+                gv[i] = v[i] * gain[c + i];
+            }
+            *reinterpret_cast<float4 *>(xr) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4 *>(xr + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            if (valid && exit_buf) {
+                float *e = exit_buf + ((size_t)b * a.max_rows + sh.dst[b] + j) * m.d + c;
+                *reinterpret_cast<float4 *>(e) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            }
+            if (valid && hidden_out) {
+                float *e = hidden_out + ((size_t)b * a.max_rows + j) * m.d + c;
+                *reinterpret_cast<float4 *>(e) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            }
+            store8_hilo(m.act_d + (size_t)t * m.d + c, m.act_d + ((size_t)m.T_alloc + t) * m.d + c, gv, m.plain);
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) m.ssq[(size_t)t * nch + ch] = ss;
+    }
+}
+
+// 1 / rms of row t, lanes fetching the chunk sums in parallel (nch <= 32); same value in every lane
+__device__ __forceinline__ float mega_inv_rms_warp(const MegaArgs &m, int t, int lane) {
+    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
+    if (nch > 32) return mega_inv_rms(m, t);
+    float s = lane < nch ? m.ssq[(size_t)t * nch + lane] : 0.f;
+    s = warp_sum(s);
+    return rsqrtf(s / (float)m.d + m.eps);
+}
+
+// a3: q,k,v = projection / rms; rotate q,k; append K,V to the sequence's pages.  One warp per (row, head).
+__device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int pool_layer, int gw, int ngw, int lane) {
+    const StageArgs &a = m.a;
+    const int hd = m.hd, half = hd / 2, heads = m.hq + 2 * m.hkv, nq = m.hq * hd;
+    const size_t stride = (size_t)m.T_pad * g.N;
+    for (int item = gw; item < m.T_pad * heads; item += ngw) {
+        const int t = item / heads, h = item % heads, b = t / a.R_pad, j = t % a.R_pad;
+        if (j >= sh.nr[b]) {
+            if (h < m.hq)
+                for (int i = lane; i < hd; i += 32) m.q[(size_t)t * nq + h * hd + i] = 0.f;
+            continue;
+        }
+        const float inv = mega_inv_rms_warp(m, t, lane);
+        const int pos = sh.p0[b] + j;
+        const int lp = pos / a.page_size, slot = pos % a.page_size;
+        const long long page = m.block_table[(size_t)b * a.max_pages + lp];
+        const bool page_ok = page >= 0 && page < m.n_pages;
+        if (!page_ok && lane == 0 && h == m.hq) atomicOr(m.status, HISPEC_ST_BOUNDS);
+        const size_t page_base = (((size_t)pool_layer * m.n_pages + (page_ok ? page : 0)) * m.hkv) * a.page_size * hd;
+        // a head's columns lie in one 128-row weight tile (head_dim 64 or 128): one slot range for the item
+        int first, ns;
+        mega_slots((h * hd) / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
+        const float *pr = m.part + (size_t)t * g.N + h * hd;
+        if (h < m.hq + m.hkv) {
+            for (int i = lane; i < half; i += 32) {
+                float x0 = 0.f, x1 = 0.f;
+                for (int s = 0; s < ns; ++s) { x0 += pr[s * stride + i]; x1 += pr[s * stride + i + half]; }
+                x0 *= inv; x1 *= inv;
+                double sn, cs;
+                sincos((double)pos * m.inv_freq[i], &sn, &cs);
+                const float c = (float)cs, sf = (float)sn;
+                const float r0 = x0 * c - x1 * sf, r1 = x1 * c + x0 * sf;
+                if (h < m.hq) {
+                    m.q[(size_t)t * nq + h * hd + i] = r0;
+                    m.q[(size_t)t * nq + h * hd + i + half] = r1;
+                } else if (page_ok) {
+                    const size_t o = page_base + ((size_t)(h - m.hq) * a.page_size + slot) * hd;
+                    m.k_pages[o + i] = __float2bfloat16_rn(r0);
+                    m.k_pages[o + i + half] = __float2bfloat16_rn(r1);
+                }
+            }
+        } else if (page_ok) {
+            const int vh = h - m.hq - m.hkv;
+            const size_t o = page_base + ((size_t)vh * a.page_size + slot) * hd;
+            for (int i = lane; i < hd; i += 32) {
+                float v = 0.f;
+                for (int s = 0; s < ns; ++s) v += pr[s * stride + i];
+                m.v_pages[o + i] = __float2bfloat16_rn(inv * v);
+            }
+        }
+    }
+}
+
+// a6 epilogue: act_f <- hi/lo( SiLU(gate / rms) * (up / rms) )
+__device__ void ew_silu(const MegaArgs &m, const MegaGemm &g, int gw, int ngw, int lane) {
+    const int nch = (m.ffn + kEwChunk - 1) / kEwChunk;
+    for (int item = gw; item < m.T_pad * nch; item += ngw) {
+        const int t = item / nch, ch = item % nch;
+        const int c = ch * kEwChunk + lane * 8;
+        const float inv = mega_inv_rms_warp(m, t, lane);
+        if (c >= m.ffn) continue;
+        float gt[8], up[8], v[8];
+        sum_slots8(m, g, t, c, gt);
+        sum_slots8(m, g, t, m.ffn + c, up);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float gg = gt[i] * inv;
+            v[i] = (gg / (1.0f + expf(-gg))) * (up[i] * inv);
+        }
+        store8_hilo(m.act_f + (size_t)t * m.ffn + c, m.act_f + ((size_t)m.T_alloc + t) * m.ffn + c, v, m.plain);
+    }
+}
+
+// a4 (second half): combine the key splits of every (row, q head) in split order -> act_o hi/lo.
+// One warp per (row, head): lanes first fetch the splits' (max, sum) pairs in parallel, then walk the
+// splits in order with the weights broadcast by shuffle, so no load waits on a branch.
+template <int HD>
+__device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw, int lane) {
+    constexpr int E = HD / 32;
+    const StageArgs &a = m.a;
+    const int nq = m.hq * HD;
+    for (int item = gw; item < m.T_pad * m.hq; item += ngw) {
+        const int t = item / m.hq, h = item % m.hq, b = t / a.R_pad, j = t % a.R_pad;
+        float acc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = 0.f;
+        float inv = 0.f;
+        if (j < sh.nr[b]) {
+            const float *base = m.attn_part + ((size_t)t * m.hq + h) * m.n_splits * (HD + 2);
+            float ms[2], ls[2];   // splits lane and lane + 32 (n_splits <= 64)
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int sidx = lane + 32 * u;
+                ms[u] = -INFINITY; ls[u] = 0.f;
+                if (sidx < m.n_splits) {
+                    ms[u] = base[(size_t)sidx * (HD + 2) + HD];
+                    ls[u] = base[(size_t)sidx * (HD + 2) + HD + 1];
+                    if (!(ls[u] > 0.f)) { ms[u] = -INFINITY; ls[u] = 0.f; }
+                }
+            }
+            float M = fmaxf(ms[0], ms[1]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+            float wv[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) wv[u] = (ms[u] == -INFINITY) ? 0.f : exp2f(ms[u] - M);
+            float L = 0.f;
+            for (int s0 = 0; s0 < m.n_splits; s0 += 8) {
+                float rv[8][E];   // issue the loads of eight splits before using any of them
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int sidx = s0 + u < m.n_splits ? s0 + u : m.n_splits - 1;
+                    const float *r = base + (size_t)sidx * (HD + 2) + lane * E;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) rv[u][e] = r[e];
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int sidx = s0 + u;
+                    if (sidx >= m.n_splits) break;
+                    const float w = __shfl_sync(0xffffffffu, wv[sidx >> 5], sidx & 31);
+                    const float l = __shfl_sync(0xffffffffu, ls[sidx >> 5], sidx & 31);
+                    L += l * w;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[e] += w * rv[u][e];
+                }
+            }
+            inv = L > 0.f ? 1.0f / L : 0.f;
+        }
+        __nv_bfloat16 *ohi = m.act_o + (size_t)t * nq + h * HD + lane * E;
+        __nv_bfloat16 *olo = m.act_o + ((size_t)m.T_alloc + t) * nq + h * HD + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) split_hi_lo(acc[e] * inv, ohi[e], olo[e], m.plain);
+    }
+}
+
+// ---- attention phase: items (split, kv head x row group, sequence) dealt round-robin to CTAs -------
+template <int HD>
+__device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, const MegaArgs &m, MegaShared &sh,
+                               uint32_t sm_attn, int pool_layer, uint32_t &pg_it, int warp, int lane) {
+    constexpr int HALVES = HD / 64, TILE = 16 * HD * 2, KS = HD / 16, NT = HD / 8;
+    const StageArgs &a = m.a;
+    volatile int *abort_flag = &sh.abort_flag;
+    const int per_b = m.n_splits * m.hkv * m.n_mg;
+    const int n_items = per_b * a.batch;
+    const int QR = m.G * a.R_pad;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int b = item / per_b, rest = item % per_b;
+        const int y = rest / m.n_splits, split = rest % m.n_splits;
+        const int kvh = y / m.n_mg, mg = y % m.n_mg;
+        const int nr = sh.nr[b], p0 = sh.p0[b];
+        const int total_pages = (p0 + nr + 15) >> 4;
+        int chunk = (total_pages + m.n_splits - 1) / m.n_splits;
+        if (chunk < 1) chunk = 1;
+        const int pg0 = split * chunk, pg1 = min(pg0 + chunk, total_pages);
+        const int n_pg = (nr > 0 && pg1 > pg0) ? pg1 - pg0 : 0;
+        if (warp == 5) {
+            for (int i0 = 0; i0 < n_pg; i0 += 32) {
+                const int my = i0 + lane;
+                long long pgid = 0;
+                if (my < n_pg) pgid = m.block_table[(size_t)b * a.max_pages + pg0 + my];
+                if (my < n_pg && (pgid < 0 || pgid >= m.n_pages)) { atomicOr(m.status, HISPEC_ST_BOUNDS); pgid = 0; }
+                const int cnt = min(32, n_pg - i0);
+                for (int u = 0; u < cnt; ++u) {
+                    const long long page = __shfl_sync(0xffffffffu, pgid, u);
+                    const uint32_t it = pg_it + i0 + u;
+                    const int s = it % kAttnStages;
+                    const uint32_t ph = (it / kAttnStages) & 1u;
+                    if (lane == 0 && a_wait(a_smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, m.status)) {
+                        const uint32_t fb = a_smem_u32(&sh.a_full[s]);
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(2 * TILE) : "memory");
+                        const int row = (int)((((long long)pool_layer * m.n_pages + page) * m.hkv + kvh) * 16);
+                        const uint32_t dk = sm_attn + s * 2 * TILE, dv = dk + TILE;
+#pragma unroll
+                        for (int h = 0; h < HALVES; ++h) {
+                            tma_load_2d(dk + h * 2048, tmK, h * 64, row, fb);
+                            tma_load_2d(dv + h * 2048, tmV, h * 64, row, fb);
+                        }
+                    }
+                }
+            }
+        } else if (warp >= 6) {
+            const int cw = warp - 6;
+            const int r_lo = mg * 64 + cw * 16 + (lane >> 2), r_hi = r_lo + 8;
+            const int j_lo = r_lo / m.G, g_lo = r_lo % m.G, j_hi = r_hi / m.G, g_hi = r_hi % m.G;
+            const bool v_lo = cw < m.mt && r_lo < QR && j_lo < nr, v_hi = cw < m.mt && r_hi < QR && j_hi < nr;
+            const int kmax_lo = v_lo ? p0 + j_lo : -1, kmax_hi = v_hi ? p0 + j_hi : -1;
+            const int nq = m.hq * HD;
+            const float *q_lo = m.q + ((size_t)(b * a.R_pad + j_lo) * nq + (size_t)(kvh * m.G + g_lo) * HD);
+            const float *q_hi = m.q + ((size_t)(b * a.R_pad + j_hi) * nq + (size_t)(kvh * m.G + g_hi) * HD);
+            uint32_t qh[KS][4], ql[KS][4];
+            const int c2 = (lane & 3) * 2;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+                for (int part = 0; part < 4; ++part) {
+                    const bool hi_row = part & 1;
+                    const float *src = hi_row ? q_hi : q_lo;
+                    const bool valid = hi_row ? v_hi : v_lo;
+                    const int col = ks * 16 + c2 + ((part & 2) ? 8 : 0);
+                    float x0 = 0.f, x1 = 0.f;
+                    if (valid) { float2 tt = *reinterpret_cast<const float2 *>(src + col); x0 = tt.x * m.scale_log2; x1 = tt.y * m.scale_log2; }
+                    const float h0 = __bfloat162float(__float2bfloat16_rn(x0)), h1 = __bfloat162float(__float2bfloat16_rn(x1));
+                    qh[ks][part] = pack_bf16(x0, x1);
+                    ql[ks][part] = pack_bf16(x0 - h0, x1 - h1);
+                }
+            }
+            float o[NT][4];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+            float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+            bool ok = true;
+            const bool active = cw < m.mt;   // warps without rows only keep the page ring moving
+            for (int i = 0; i < n_pg && ok; ++i) {
+                const uint32_t it = pg_it + i;
+                const int s = it % kAttnStages;
+                const uint32_t ph = (it / kAttnStages) & 1u;
+                ok = a_wait(a_smem_u32(&sh.a_full[s]), ph, abort_flag, m.status);
+                if (!ok) break;
+                if (active) {
+                    const uint32_t sk = sm_attn + s * 2 * TILE, sv = sk + TILE;
+                    float sc[2][4];
+#pragma unroll
+                    for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+                    const int mat = lane >> 3, rin = lane & 7;
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        const int key = (mat >> 1) * 8 + rin;
+                        const int chunk16 = (ks & 3) * 2 + (mat & 1);
+                        const uint32_t addr = sk + (ks >> 2) * 2048 + key * 128 + ((chunk16 ^ (key & 7)) << 4);
+                        uint32_t kb[4];
+                        ldmatrix_x4(addr, kb);
+                        mma_bf16_16816(sc[0], qh[ks], kb[0], kb[1]);
+                        mma_bf16_16816(sc[0], ql[ks], kb[0], kb[1]);
+                        mma_bf16_16816(sc[1], qh[ks], kb[2], kb[3]);
+                        mma_bf16_16816(sc[1], ql[ks], kb[2], kb[3]);
+                    }
+                    const int key0 = (pg0 + i) * 16;
+                    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int key = key0 + n * 8 + c2 + e;
+                            if (key > kmax_lo) sc[n][e] = -INFINITY;
+                            if (key > kmax_hi) sc[n][2 + e] = -INFINITY;
+                            mx_lo = fmaxf(mx_lo, sc[n][e]);
+                            mx_hi = fmaxf(mx_hi, sc[n][2 + e]);
+                        }
+                    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+                    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+                    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+                    const float base_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, base_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+                    const float cr_lo = exp2f(m_lo - base_lo), cr_hi = exp2f(m_hi - base_hi);
+                    m_lo = mn_lo; m_hi = mn_hi;
+                    const float e00 = exp2f(sc[0][0] - base_lo), e01 = exp2f(sc[0][1] - base_lo);
+                    const float e02 = exp2f(sc[0][2] - base_hi), e03 = exp2f(sc[0][3] - base_hi);
+                    const float e10 = exp2f(sc[1][0] - base_lo), e11 = exp2f(sc[1][1] - base_lo);
+                    const float e12 = exp2f(sc[1][2] - base_hi), e13 = exp2f(sc[1][3] - base_hi);
+                    uint32_t pa[4] = {pack_bf16(e00, e01), pack_bf16(e02, e03), pack_bf16(e10, e11), pack_bf16(e12, e13)};
+                    l_lo = l_lo * cr_lo + (e00 + e01 + e10 + e11);
+                    l_hi = l_hi * cr_hi + (e02 + e03 + e12 + e13);
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) { o[n][0] *= cr_lo; o[n][1] *= cr_lo; o[n][2] *= cr_hi; o[n][3] *= cr_hi; }
+#pragma unroll
+                    for (int n = 0; n < NT; n += 2) {
+                        const int key = (mat & 1) * 8 + rin;
+                        const int cg = n + (mat >> 1);
+                        const uint32_t addr = sv + (cg >> 3) * 2048 + key * 128 + (((cg & 7) ^ (key & 7)) << 4);
+                        uint32_t vb[4];
+                        ldmatrix_x4_trans(addr, vb);
+                        mma_bf16_16816(o[n], pa, vb[0], vb[1]);
+                        mma_bf16_16816(o[n + 1], pa, vb[2], vb[3]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(&sh.a_empty[s])) : "memory");
+            }
+            l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+            l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+            l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+            l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+            if (!ok) { l_lo = l_hi = 0.f; m_lo = m_hi = -INFINITY; }
+            if (v_lo) {
+                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_lo) * m.hq + kvh * m.G + g_lo) * m.n_splits + split) * (HD + 2));
+#pragma unroll
+                for (int n = 0; n < NT; ++n) *reinterpret_cast<float2 *>(dst + n * 8 + c2) = make_float2(o[n][0], o[n][1]);
+                if ((lane & 3) == 0) { dst[HD] = m_lo; dst[HD + 1] = l_lo; }
+            }
+            if (v_hi) {
+                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_hi) * m.hq + kvh * m.G + g_hi) * m.n_splits + split) * (HD + 2));
+#pragma unroll
+                for (int n = 0; n < NT; ++n) *reinterpret_cast<float2 *>(dst + n * 8 + c2) = make_float2(o[n][2], o[n][3]);
+                if ((lane & 3) == 0) { dst[HD] = m_hi; dst[HD + 1] = l_hi; }
+            }
+        }
+        pg_it += n_pg;
+    }
+}
+
+// ---- projection phase roles -----------------------------------------------------------------
+struct MegaRing {
+    uint32_t base;         // shared address of stage 0 of this pipeline
+    uint32_t stage_bytes;  // 16 KiB weight tile + activation tile
+    uint32_t x_bytes;
+    int stages;
+};
+
+// position in the call's flattened sequence of weight blocks (projection, tile, k-block) of one pipeline
+struct WCursor {
+    const MegaArgs *m;
+    int p;
+    int gi, n_g;   // projection index in call order; 4 per layer, then the exit head
+    SegIter seg;
+    int tile, kb, kb1;
+    bool valid;
+    __device__ const MegaGemm *gemm() const {
+        return gi + 1 < n_g ? &m->gemms[(m->a.l0 + gi / 4) * 4 + (gi & 3)] : m->head;
+    }
+    __device__ WCursor(const MegaArgs *m_, int p_)
+        : m(m_), p(p_), gi(-1), n_g(4 * (m_->a.l1 - m_->a.l0) + 1), seg(1, 1, 0, 0, 0, 1), tile(0), kb(0), kb1(0), valid(true) {
+        seg.u = seg.hi = 0;
+        advance();
+    }
+    __device__ void advance() {
+        if (++kb < kb1) return;
+        int kb0;
+        while (!seg.next(tile, kb0, kb1)) {
+            if (++gi >= n_g) { valid = false; return; }
+            const MegaGemm *g = gemm();
+            seg = SegIter(g->tiles, g->kb_total, gi + 1 == n_g, blockIdx.x, p, gridDim.x);
+        }
+        kb = kb0;
+    }
+};
+
+// warps 0 and 1, one thread each: every weight block of the call that belongs to pipeline p, in
+// consumption order, into that pipeline's ring -- across projection and phase boundaries
+__device__ __forceinline__ void mega_w_producer(const MegaArgs &m, int p, const MegaRing &ring, MegaShared &sh) {
+    volatile int *ab = &sh.abort_flag;
+    WCursor ld(&m, p);
+    uint32_t it = 0;
+    while (ld.valid) {
+        const int s = it % ring.stages;
+        const uint32_t ph = (it / ring.stages) & 1u;
+        if (!mbar_wait(smem_u32(&sh.empty[p][s]), ph ^ 1u, ab, m.status)) return;
+        const uint32_t fb = smem_u32(&sh.w_full[p][s]);
+        mbar_expect_tx(fb, kWTileBytes);
+        const MegaGemm *g = ld.gemm();
+        tma_load_2d(ring.base + s * ring.stage_bytes, &g->tmW, ld.kb * kTileK, ld.tile * kWeightTileRows, fb);
+        ld.advance();
+        ++it;
+    }
+}
+
+__device__ __forceinline__ bool mega_x_load(const MegaGemm *g, int whole, int p, const CUtensorMap *tmX,
+                                            const MegaRing &ring, MegaShared &sh, uint32_t &it, uint32_t *status) {
+    volatile int *ab = &sh.abort_flag;
+    SegIter seg(g->tiles, g->kb_total, whole, blockIdx.x, p, gridDim.x);
+    int tile, kb0, kb1;
+    while (seg.next(tile, kb0, kb1)) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            const int s = it % ring.stages;
+            const uint32_t ph = (it / ring.stages) & 1u;
+            if (!mbar_wait(smem_u32(&sh.empty[p][s]), ph ^ 1u, ab, status)) return false;
+            const uint32_t fb = smem_u32(&sh.x_full[p][s]);
+            mbar_expect_tx(fb, ring.x_bytes);
+            tma_load_3d(ring.base + s * ring.stage_bytes + kWTileBytes, tmX, kb * kTileK, 0, 0, fb);
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ bool mega_mma(const MegaGemm *g, int whole, int p, int ncols, const MegaRing &ring,
+                                         MegaShared &sh, uint32_t &it, uint32_t &seg_it, uint32_t *status) {
+    volatile int *ab = &sh.abort_flag;
+    const uint32_t idesc = umma_idesc_bf16(ncols);
+    SegIter seg(g->tiles, g->kb_total, whole, blockIdx.x, p, gridDim.x);
+    int tile, kb0, kb1;
+    while (seg.next(tile, kb0, kb1)) {
+        const int buf = seg_it & 1;
+        const uint32_t aph = (seg_it >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&sh.acc_empty[p][buf]), aph ^ 1u, ab, status)) return false;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tmem_d = sh.tmem + (p * 2 + buf) * kMegaAccCols;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            const int s = it % ring.stages;
+            const uint32_t ph = (it / ring.stages) & 1u;
+            if (!mbar_wait(smem_u32(&sh.w_full[p][s]), ph, ab, status)) return false;
+            if (!mbar_wait(smem_u32(&sh.x_full[p][s]), ph, ab, status)) return false;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t ad = umma_desc_sw128(ring.base + s * ring.stage_bytes);
+            const uint64_t bd = umma_desc_sw128(ring.base + s * ring.stage_bytes + kWTileBytes);
+#pragma unroll
+            for (int k = 0; k < kTileK / 16; ++k)
+                umma_bf16(tmem_d, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), idesc, (kb > kb0 || k) ? 1u : 0u);
+            umma_commit(smem_u32(&sh.empty[p][s]));
+        }
+        umma_commit(smem_u32(&sh.acc_full[p][buf]));
+        ++seg_it;
+    }
+    return true;
+}
+
+// accumulator columns [c0, c0 + 8) of this warp's 32 TMEM lanes, hi + lo planes added
+__device__ __forceinline__ void mega_acc_ld8(uint32_t taddr, int c0, int t_box, int planes, float *v) {
+    tmem_ld8(taddr + (uint32_t)c0, v);
+    if (planes == 2) {
+        float w[8];
+        tmem_ld8(taddr + (uint32_t)(t_box + c0), w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] += w[i];
+    }
+}
+
+// warps 6..9, split-K projections: drain the accumulators of both pipelines' segments, alternating
+__device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, const MegaArgs &m, MegaShared &sh,
+                                                   uint32_t *seg_it, int warp, int lane) {
+    volatile int *ab = &sh.abort_flag;
+    const int lg = warp & 3;
+    SegIter seg0(g->tiles, g->kb_total, 0, blockIdx.x, 0, gridDim.x), seg1(g->tiles, g->kb_total, 0, blockIdx.x, 1, gridDim.x);
+    const size_t stride = (size_t)m.T_pad * g->N;
+    bool more0 = true, more1 = true;
+    while (more0 || more1) {
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            int tile, kb0, kb1;
+            bool has = p ? (more1 && (more1 = seg1.next(tile, kb0, kb1))) : (more0 && (more0 = seg0.next(tile, kb0, kb1)));
+            if (!has) continue;
+            const int buf = seg_it[p] & 1;
+            const uint32_t aph = (seg_it[p] >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&sh.acc_full[p][buf]), aph, ab, m.status)) return false;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t taddr = sh.tmem + (p * 2 + buf) * kMegaAccCols + ((uint32_t)(lg * 32) << 16);
+            const int n = tile * kWeightTileRows + lg * 32 + lane;
+            int first, ns;
+            mega_slots(tile, g->tiles, g->kb_total, gridDim.x, first, ns);
+            const int slot = 2 * blockIdx.x + p - first;
+            for (int c0 = 0; c0 < m.T_pad; c0 += 8) {
+                float v[8];
+                mega_acc_ld8(taddr, c0, m.t_box, m.planes, v);
+                if (n < g->N) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (c0 + i < m.T_pad) m.part[slot * stride + (size_t)(c0 + i) * g->N + n] = v[i];
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&sh.acc_empty[p][buf])) : "memory");
+            ++seg_it[p];
+        }
+    }
+    return true;
+}
+
+// warps 6..9, exit head: each tile's accumulator is the sum of the two pipelines' K halves; every
+// column (activation row) is reduced to its top-2 over this warp's 32 vocabulary entries
+__device__ __forceinline__ bool mega_epilogue_head(const MegaGemm *g, const MegaArgs &m, MegaShared &sh,
+                                                   uint32_t *seg_it, int warp, int lane) {
+    volatile int *ab = &sh.abort_flag;
+    const int lg = warp & 3;
+    SegIter seg(g->tiles, g->kb_total, 1, blockIdx.x, 0, gridDim.x);
+    int tile, kb0, kb1;
+    while (seg.next(tile, kb0, kb1)) {
+        uint32_t taddr[2];
+        int bufs[2];
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            bufs[p] = seg_it[p] & 1;
+            const uint32_t aph = (seg_it[p] >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&sh.acc_full[p][bufs[p]]), aph, ab, m.status)) return false;
+            taddr[p] = sh.tmem + (p * 2 + bufs[p]) * kMegaAccCols + ((uint32_t)(lg * 32) << 16);
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int n = tile * kWeightTileRows + lg * 32 + lane;
+        for (int c0 = 0; c0 < m.T_pad; c0 += 8) {
+            float v[8], w[8];
+            mega_acc_ld8(taddr[0], c0, m.t_box, m.planes, v);
+            mega_acc_ld8(taddr[1], c0, m.t_box, m.planes, w);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (c0 + i >= m.T_pad) break;
+                const int t = c0 + i;
+                const float val = (n < g->N) ? v[i] + w[i] : -INFINITY;
+                if (m.logits && n < g->N) {
+                    const int b = t / m.a.R_pad, j = t % m.a.R_pad;
+                    if (j < sh.nr[b]) m.logits[((size_t)b * m.a.max_rows + j) * g->N + n] = val * mega_inv_rms(m, t);
+                }
+                Top2 best = top2_warp(Top2{val, -INFINITY, n < g->N ? n : 0x7fffffff});
+                if (lane == 0) {
+                    float *o = m.top_part + ((size_t)(tile * 4 + lg) * m.T_pad + t) * 4;
+                    o[0] = best.v1; o[1] = __int_as_float(best.i1); o[2] = best.v2;
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&sh.acc_empty[p][bufs[p]])) : "memory");
+            ++seg_it[p];
+        }
+    }
+    return true;
+}
+
+// ---- a9 (second half) + a10 for sequence b, by the worker threads of one CTA ---------------------
+__device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b) {
+    const StageArgs &a = m.a;
+    const AcceptArgs &r = m.r;
+    const int nr = sh.nr[b];
+    const int wt = threadIdx.x - kMegaLeader, lane = threadIdx.x & 31, w = (threadIdx.x >> 5) - 2;
+    const int n_rec = m.head->tiles * 4;
+    for (int j = 0; j < nr; ++j) {
+        const int t = b * a.R_pad + j;
+        Top2 best = {-INFINITY, -INFINITY, 0x7fffffff};
+        for (int rec = wt; rec < n_rec; rec += kMegaWorkers) {
+            const float *o = m.top_part + ((size_t)rec * m.T_pad + t) * 4;
+            best = top2_merge(best, Top2{o[0], o[2], __float_as_int(o[1])});
+        }
+        best = top2_warp(best);
+        worker_bar();
+        if (lane == 0) { sh.red_v1[w] = best.v1; sh.red_v2[w] = best.v2; sh.red_i1[w] = best.i1; }
+        worker_bar();
+        if (threadIdx.x == kMegaLeader) {
+            Top2 mm = {sh.red_v1[0], sh.red_v2[0], sh.red_i1[0]};
+            for (int i = 1; i < kMegaWorkers / 32; ++i) mm = top2_merge(mm, Top2{sh.red_v1[i], sh.red_v2[i], sh.red_i1[i]});
+            const float inv = mega_inv_rms(m, t);
+            m.argmax_ws[t] = mm.i1;
+            if (r.argmax_ids) r.argmax_ids[(size_t)b * a.max_rows + j] = mm.i1;
+            if (r.top2) {
+                r.top2[((size_t)b * a.max_rows + j) * 2] = mm.v1 * inv;
+                r.top2[((size_t)b * a.max_rows + j) * 2 + 1] = mm.v2 * inv;
+            }
+        }
+    }
+    worker_bar();
+    if (threadIdx.x != kMegaLeader) return;
+    const int p0 = sh.p0[b];
+    if (a.mode == 1) {
+        const int nd = sh.nd[b];
+        int acc = 0;
+        while (acc < nd && acc < nr && r.draft_tokens[(size_t)b * r.token_stride + acc] == m.argmax_ws[b * a.R_pad + acc]) ++acc;
+        if (r.n_accepted) r.n_accepted[b] = acc;
+        if (r.next_token) r.next_token[b] = (acc < nr) ? m.argmax_ws[b * a.R_pad + acc] : -1;
+        if (r.pending && nr > 0) {
+            if (acc < nr) r.pending[b] = m.argmax_ws[b * a.R_pad + acc];
+            else if (acc > 0) r.pending[b] = r.draft_tokens[(size_t)b * r.token_stride + acc - 1];
+        }
+        if (r.tentative && a.l1 == a.L_i && nr > 0) {
+            int32_t *tv = r.tentative + (size_t)b * a.max_rows + sh.dst[b];
+            for (int j = 0; j < acc; ++j) tv[j] = r.draft_tokens[(size_t)b * r.token_stride + j];
+            if (acc < nr) tv[acc] = m.argmax_ws[b * a.R_pad + acc];
+        }
+        if (nr > 0) {
+            const int nl = p0 + min(acc + 1, nr);
+            m.len_d[b] = nl;
+            if (a.l1 > a.L_d) m.len_i[b] = nl;
+            if (a.l1 > a.L_i) m.len_f[b] = nl;
+        }
+    } else if (nr > 0) {
+        const int nl = p0 + nr;
+        m.len_d[b] = nl;
+        if (a.l1 > a.L_d) m.len_i[b] = nl;
+        if (a.l1 > a.L_i) m.len_f[b] = nl;
+        if (r.out_tokens) {
+            bool emit = true;
+            if (r.n_tokens) emit = (nl == r.n_tokens[b]);
+            if (emit) r.out_tokens[(size_t)b * r.out_stride] = m.argmax_ws[b * a.R_pad + nr - 1];
+        }
+    }
+}
+
+// ---- the kernel --------------------------------------------------------------------------------
+template <int HD>
+__global__ void __launch_bounds__(kMegaThreads, 1)
+hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_constant__ CUtensorMap tmXo,
+                    const __grid_constant__ CUtensorMap tmXf, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ MegaArgs m) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ MegaShared sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const StageArgs &a = m.a;
+    const int ncols = m.t_box * m.planes;
+
+    MegaRing ring[2];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    for (int p = 0; p < 2; ++p) {
+        ring[p].x_bytes = (uint32_t)ncols * 128u;
+        ring[p].stage_bytes = kWTileBytes + ring[p].x_bytes;
+        ring[p].stages = m.stages;
+        ring[p].base = base + p * m.stages * ring[p].stage_bytes;
+    }
+    const uint32_t sm_attn = base + 2 * m.stages * ring[0].stage_bytes;  // 1024-aligned: stage_bytes is a multiple of 2048
+
+    if (threadIdx.x == 0) {
+        sh.abort_flag = 0;
+        sh.trace_n = 0;
+        sh.bar_k = 0;
+        if (blockIdx.x == 0) *((volatile unsigned *)m.bar_next) = 0u;
+        if (m.trace && blockIdx.x == 0) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+            m.trace[1023] = t;
+        }
+        for (int p = 0; p < 2; ++p) {
+            for (int s = 0; s < m.stages; ++s) {
+                mbar_init(smem_u32(&sh.w_full[p][s]), 1);
+                mbar_init(smem_u32(&sh.x_full[p][s]), 1);
+                mbar_init(smem_u32(&sh.empty[p][s]), 1);
+            }
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(smem_u32(&sh.acc_full[p][i]), 1);
+                mbar_init(smem_u32(&sh.acc_empty[p][i]), 4);
+            }
+        }
+        for (int s = 0; s < kAttnStages; ++s) {
+            mbar_init(smem_u32(&sh.a_full[s]), 1);
+            mbar_init(smem_u32(&sh.a_empty[s]), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    mega_prep_rows(m, sh);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+    if (warp < 2) {
+        // ---- weight producers: the whole call's weight blocks of pipeline `warp`, in consumption order
+        if (lane == 0) mega_w_producer(m, warp, ring[warp], sh);
+    } else {
+        const int gw = (warp - 2) * gridDim.x + blockIdx.x, ngw = (kMegaWorkers / 32) * gridDim.x;
+        uint32_t it = 0, seg_it[2] = {0, 0}, pg_it = 0;   // per-thread progress counters of the role loops
+        const CUtensorMap *tmX[3] = {&tmXd, &tmXo, &tmXf};
+        auto gemm_phase = [&](const MegaGemm *g, int whole, int xbuf) {
+            if (warp == 2 || warp == 3) {
+                const int p = warp - 2;
+                if (lane == 0) mega_mma(g, whole, p, ncols, ring[p], sh, it, seg_it[p], m.status);
+            } else if (warp == 4 || warp == 5) {
+                const int p = warp - 4;
+                if (lane == 0) mega_x_load(g, whole, p, tmX[xbuf], ring[p], sh, it, m.status);
+            } else {
+                if (whole) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
+                else mega_epilogue_part(g, m, sh, seg_it, warp, lane);
+            }
+            grid_sync(m, sh);
+        };
+        ew_rows_in(m, sh, m.attn_norm[a.l0], gw, ngw, lane);
+        grid_sync(m, sh);
+        for (int l = a.l0; l < a.l1; ++l) {
+            const MegaGemm *G4 = &m.gemms[l * 4];
+            const int pool_layer = l - m.first_layer;
+            gemm_phase(&G4[0], 0, 0);
+            ew_qkv(m, sh, G4[0], pool_layer, gw, ngw, lane);
+            grid_sync(m, sh);
+            mega_attention<HD>(&tmK, &tmV, m, sh, sm_attn, pool_layer, pg_it, warp, lane);
+            grid_sync(m, sh);
+            ew_attn_merge<HD>(m, sh, gw, ngw, lane);
+            grid_sync(m, sh);
+            gemm_phase(&G4[1], 0, 1);
+            ew_resid(m, sh, G4[1], m.ffn_norm[l], nullptr, nullptr, gw, ngw, lane);
+            grid_sync(m, sh);
+            gemm_phase(&G4[2], 0, 0);
+            ew_silu(m, G4[2], gw, ngw, lane);
+            grid_sync(m, sh);
+            gemm_phase(&G4[3], 0, 2);
+            const bool last = l + 1 == a.l1;
+            ew_resid(m, sh, G4[3], last ? m.final_norm : m.attn_norm[l + 1], last ? m.exit_buf : nullptr,
+                     last ? m.hidden_out : nullptr, gw, ngw, lane);
+            grid_sync(m, sh);
+        }
+        gemm_phase(m.head, 1, 0);
+        for (int b = blockIdx.x; b < a.batch; b += gridDim.x) mega_accept(m, sh, b);
+    }
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh.tmem), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace hispec

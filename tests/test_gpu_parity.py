@@ -17,7 +17,7 @@ from tests.helpers import oracle_for
 
 pytestmark = pytest.mark.gpu
 
-FLAG_SETS = {"tcgen05": 0, "simt": 1, "tcgen05-plain": 2, "rowwarp-attn": 8}
+FLAG_SETS = {"tcgen05": 0, "simt": 1, "tcgen05-plain": 2, "rowwarp-attn": 8, "multi-kernel": 16}
 
 
 def _binding():
@@ -103,7 +103,7 @@ def _tiny_setup(flags, n_prompt, n_gen, N_d, rounds, resid_scale=None):
     return shape, w, m, hs, ctx, st, max_rows
 
 
-@pytest.mark.parametrize("flagname", ["simt", "tcgen05", "tcgen05-plain", "rowwarp-attn"])
+@pytest.mark.parametrize("flagname", ["simt", "tcgen05", "tcgen05-plain", "rowwarp-attn", "multi-kernel"])
 def test_tiny_config_every_call(flagname):
     """cfg "tiny" as stated: prompt 128, k = 4 greedy drafts from the draft exit, target every 2
     rounds, 64 generated tokens -- every draft / verify-I / verify-T call compared."""
@@ -177,7 +177,7 @@ def test_tiny_prefill_and_free_running_lossless():
     ctx.close(); ctx2.close()
 
 
-@pytest.mark.parametrize("flagname", ["tcgen05", "simt", "rowwarp-attn"])
+@pytest.mark.parametrize("flagname", ["tcgen05", "simt", "rowwarp-attn", "multi-kernel"])
 def test_batched_ragged_gqa_pages_permuted(flagname):
     """GQA 2:1, head_dim 128, odd sizes (d 320, ffn 400, vocab 1000): a batch of 3 sequences with different
     context lengths, ragged row counts and scattered pages against the oracle, one sequence at a time;
