@@ -38,8 +38,8 @@ METRIC = "verified tokens/s per B200 (HiSpec, Llama-3-8B shape, batch 1, k=5)"
 UNIT = "tokens/s"
 N_PROMPT, N_D, ROUNDS = 1024, 5, 2
 # dram__bytes_read.sum + dram__bytes_write.sum of one hispec_stage_kernel launch (a verify-I call of this
-# workload) from the ncu capture summarised under profiles/; None until a capture exists
-ROOFLINE_TRAFFIC_BYTES_PER_LAUNCH = None
+# workload: layers [8,16) + head, 6 rows, context 1024) from the ncu capture summarised under profiles/
+ROOFLINE_TRAFFIC_BYTES_PER_LAUNCH = 4.687e9
 
 
 def peaks():
