@@ -184,23 +184,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             for (int i = 0; i < pre; ++i)
                 tma_load_3d(smem0 + i * stage_bytes + kWTileBytes, &tmX, (kb0 + i) * kTileK, g.row0, 0,
                             smem_u32(&bar_full[i]));
+            int s = pre == g.stages ? 0 : pre;   // slot and phase bit advance without divisions
+            uint32_t ph = pre == g.stages ? 1u : 0u;
             for (int i = pre; i < nkb; ++i) {
-                int s = i % g.stages;
-                uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, abort_flag, g.status)) break;
                 uint32_t fb = smem_u32(&bar_full[s]);
                 mbar_expect_tx(fb, stage_bytes);
                 tma_load_2d(smem0 + s * stage_bytes, &tmW, (kb0 + i) * kTileK, tile * kWeightTileRows, fb);
                 tma_load_3d(smem0 + s * stage_bytes + kWTileBytes, &tmX, (kb0 + i) * kTileK, g.row0, 0, fb);
+                if (++s == g.stages) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(ncols);
             bool ok = true;
+            int s = 0;
+            uint32_t ph = 0;
             for (int i = 0; i < nkb && ok; ++i) {
-                int s = i % g.stages;
-                uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 ok = mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -210,6 +211,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 for (int k = 0; k < kTileK / 16; ++k)
                     umma_bf16(tmem_d, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), idesc, (i | k) ? 1u : 0u);
                 umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
+                if (++s == g.stages) { s = 0; ph ^= 1u; }
             }
             umma_commit(smem_u32(&bar_acc));           // accumulator complete
         }

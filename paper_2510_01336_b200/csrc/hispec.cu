@@ -608,8 +608,13 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     if (stages > kMegaMaxStages) stages = kMegaMaxStages;
     if (stages < 2) return 1;
     m.stages = stages;
-    for (int k = 0; k < G_HEAD; ++k)
+    for (int k = 0; k < G_HEAD; ++k) {
         if (x->mega_part_floats[k] * (size_t)T_pad > c->part_floats) return 1;
+        // the kernel's partition arithmetic is 32-bit and its per-pipeline segment lists are fixed-size
+        if ((long long)c->plan[k].tiles * c->plan[k].kb_total * 2 * c->sm_count >= (1ll << 31)) return 1;
+        if (ceil_div(ceil_div(c->plan[k].tiles * c->plan[k].kb_total, 2 * c->sm_count), c->plan[k].kb_total) + 2 > kMegaMaxSegs) return 1;
+    }
+    if (ceil_div(c->plan[G_HEAD].tiles, c->sm_count) > kMegaMaxSegs) return 1;
     m.len_d = kv.len_draft; m.len_i = kv.len_inter; m.len_f = kv.len_target;
     m.n_rows_in = sc.n_rows; m.n_draft_in = sc.n_draft; m.tokens = sc.tokens; m.n_tokens = sc.n_tokens;
     m.tok_emb = (const __nv_bfloat16 *)c->tok_emb;

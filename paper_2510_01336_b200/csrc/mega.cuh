@@ -83,7 +83,18 @@ struct MegaArgs {
     unsigned long long *trace;  // optional: CTA 0 stamps the global timer after every grid barrier
 };
 
+// Segment lists (tile, k-block range) of this CTA's two pipelines for each kind of projection, worked out
+// once at kernel start: the role loops are single threads, for which a 64-bit division costs about a
+// microsecond of pure latency.
+constexpr int kMegaMaxSegs = 16;
+struct SegList {
+    int n;
+    int tile[kMegaMaxSegs];
+    short kb0[kMegaMaxSegs], kb1[kMegaMaxSegs];
+};
+
 struct MegaShared {
+    SegList segs[5][2];      // [QKV, O, gate/up, down, head][pipeline]
     uint64_t w_full[2][kMegaMaxStages], x_full[2][kMegaMaxStages], empty[2][kMegaMaxStages];
     uint64_t acc_full[2][2], acc_empty[2][2];
     uint64_t a_full[kAttnStages], a_empty[kAttnStages];
@@ -139,10 +150,12 @@ struct SegIter {
 };
 // slots of a tile: one per CTA whose span touches it, in CTA order
 __host__ __device__ inline void mega_slots(int tile, int tiles, int kbt, int G, int &first_cta, int &n_slots) {
-    long long U = (long long)tiles * kbt;
-    int Ge = mega_eff_ctas(U, 2 * G);
-    first_cta = mega_cta_of((long long)tile * kbt, U, Ge);
-    n_slots = mega_cta_of((long long)(tile + 1) * kbt - 1, U, Ge) - first_cta + 1;
+    // 32-bit arithmetic: the host only takes this path when tiles * kbt * 2G < 2^31
+    const unsigned U = (unsigned)tiles * (unsigned)kbt;
+    const unsigned Ge = U < 2u * (unsigned)G ? U : 2u * (unsigned)G;
+    const unsigned u0 = (unsigned)tile * (unsigned)kbt, u1 = u0 + (unsigned)kbt - 1u;
+    first_cta = (int)(((u0 + 1u) * Ge + U - 1u) / U) - 1;
+    n_slots = (int)(((u1 + 1u) * Ge + U - 1u) / U) - 1 - first_cta + 1;
 }
 
 // ---- barriers --------------------------------------------------------------------------------
@@ -686,32 +699,54 @@ struct MegaRing {
     uint32_t x_bytes;
     int stages;
 };
+// slot index and phase bit of a role's running position in its ring (no division in the loops)
+struct RingPos {
+    int s;
+    uint32_t ph;
+    __device__ RingPos() : s(0), ph(0) {}
+    __device__ __forceinline__ void advance(int stages) {
+        if (++s == stages) { s = 0; ph ^= 1u; }
+    }
+};
 
-// position in the call's flattened sequence of weight blocks (projection, tile, k-block) of one pipeline
+__device__ __forceinline__ void mega_fill_seglists(const MegaArgs &m, MegaShared &sh) {
+    if (threadIdx.x >= 10) return;
+    const int kind = threadIdx.x >> 1, p = threadIdx.x & 1;
+    const MegaGemm *g = kind < 4 ? &m.gemms[m.a.l0 * 4 + kind] : m.head;
+    SegIter seg(g->tiles, g->kb_total, kind == 4, blockIdx.x, p, gridDim.x);
+    SegList &L = sh.segs[kind][p];
+    int n = 0, tile, kb0, kb1;
+    while (n < kMegaMaxSegs && seg.next(tile, kb0, kb1)) {
+        L.tile[n] = tile; L.kb0[n] = (short)kb0; L.kb1[n] = (short)kb1;
+        ++n;
+    }
+    L.n = n;
+}
+
+// position in the call's flattened sequence of weight blocks (projection, segment, k-block) of one pipeline
 struct WCursor {
     const MegaArgs *m;
+    const MegaShared *sh;
     int p;
     int gi, n_g;   // projection index in call order; 4 per layer, then the exit head
-    SegIter seg;
-    int tile, kb, kb1;
+    int si, tile, kb, kb1;
     bool valid;
+    __device__ int kind() const { return gi + 1 < n_g ? (gi & 3) : 4; }
     __device__ const MegaGemm *gemm() const {
-        return gi + 1 < n_g ? &m->gemms[(m->a.l0 + gi / 4) * 4 + (gi & 3)] : m->head;
+        return gi + 1 < n_g ? &m->gemms[(m->a.l0 + (gi >> 2)) * 4 + (gi & 3)] : m->head;
     }
-    __device__ WCursor(const MegaArgs *m_, int p_)
-        : m(m_), p(p_), gi(-1), n_g(4 * (m_->a.l1 - m_->a.l0) + 1), seg(1, 1, 0, 0, 0, 1), tile(0), kb(0), kb1(0), valid(true) {
-        seg.u = seg.hi = 0;
+    __device__ WCursor(const MegaArgs *m_, const MegaShared *sh_, int p_)
+        : m(m_), sh(sh_), p(p_), gi(0), n_g(4 * (m_->a.l1 - m_->a.l0) + 1), si(-1), tile(0), kb(0), kb1(0), valid(true) {
         advance();
     }
     __device__ void advance() {
         if (++kb < kb1) return;
-        int kb0;
-        while (!seg.next(tile, kb0, kb1)) {
+        for (;;) {
+            const SegList &L = sh->segs[kind()][p];
+            if (++si < L.n) { tile = L.tile[si]; kb = L.kb0[si]; kb1 = L.kb1[si]; return; }
+            si = -1;
             if (++gi >= n_g) { valid = false; return; }
-            const MegaGemm *g = gemm();
-            seg = SegIter(g->tiles, g->kb_total, gi + 1 == n_g, blockIdx.x, p, gridDim.x);
         }
-        kb = kb0;
     }
 };
 
@@ -719,63 +754,58 @@ struct WCursor {
 // consumption order, into that pipeline's ring -- across projection and phase boundaries
 __device__ __forceinline__ void mega_w_producer(const MegaArgs &m, int p, const MegaRing &ring, MegaShared &sh) {
     volatile int *ab = &sh.abort_flag;
-    WCursor ld(&m, p);
-    uint32_t it = 0;
+    WCursor ld(&m, &sh, p);
+    RingPos pos;
     while (ld.valid) {
-        const int s = it % ring.stages;
-        const uint32_t ph = (it / ring.stages) & 1u;
-        if (!mbar_wait(smem_u32(&sh.empty[p][s]), ph ^ 1u, ab, m.status)) return;
-        const uint32_t fb = smem_u32(&sh.w_full[p][s]);
+        if (!mbar_wait(smem_u32(&sh.empty[p][pos.s]), pos.ph ^ 1u, ab, m.status)) return;
+        const uint32_t fb = smem_u32(&sh.w_full[p][pos.s]);
         mbar_expect_tx(fb, kWTileBytes);
         const MegaGemm *g = ld.gemm();
-        tma_load_2d(ring.base + s * ring.stage_bytes, &g->tmW, ld.kb * kTileK, ld.tile * kWeightTileRows, fb);
+        tma_load_2d(ring.base + pos.s * ring.stage_bytes, &g->tmW, ld.kb * kTileK, ld.tile * kWeightTileRows, fb);
         ld.advance();
-        ++it;
+        pos.advance(ring.stages);
     }
 }
 
-__device__ __forceinline__ bool mega_x_load(const MegaGemm *g, int whole, int p, const CUtensorMap *tmX,
-                                            const MegaRing &ring, MegaShared &sh, uint32_t &it, uint32_t *status) {
+__device__ __forceinline__ bool mega_x_load(int kind, int p, const CUtensorMap *tmX, const MegaRing &ring,
+                                            MegaShared &sh, RingPos &pos, uint32_t *status) {
     volatile int *ab = &sh.abort_flag;
-    SegIter seg(g->tiles, g->kb_total, whole, blockIdx.x, p, gridDim.x);
-    int tile, kb0, kb1;
-    while (seg.next(tile, kb0, kb1)) {
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-            const int s = it % ring.stages;
-            const uint32_t ph = (it / ring.stages) & 1u;
-            if (!mbar_wait(smem_u32(&sh.empty[p][s]), ph ^ 1u, ab, status)) return false;
-            const uint32_t fb = smem_u32(&sh.x_full[p][s]);
+    const SegList &L = sh.segs[kind][p];
+    for (int i = 0; i < L.n; ++i) {
+        for (int kb = L.kb0[i]; kb < L.kb1[i]; ++kb) {
+            if (!mbar_wait(smem_u32(&sh.empty[p][pos.s]), pos.ph ^ 1u, ab, status)) return false;
+            const uint32_t fb = smem_u32(&sh.x_full[p][pos.s]);
             mbar_expect_tx(fb, ring.x_bytes);
-            tma_load_3d(ring.base + s * ring.stage_bytes + kWTileBytes, tmX, kb * kTileK, 0, 0, fb);
+            tma_load_3d(ring.base + pos.s * ring.stage_bytes + kWTileBytes, tmX, kb * kTileK, 0, 0, fb);
+            pos.advance(ring.stages);
         }
     }
     return true;
 }
 
-__device__ __forceinline__ bool mega_mma(const MegaGemm *g, int whole, int p, int ncols, const MegaRing &ring,
-                                         MegaShared &sh, uint32_t &it, uint32_t &seg_it, uint32_t *status) {
+__device__ __forceinline__ bool mega_mma(int kind, int p, int ncols, const MegaRing &ring, MegaShared &sh,
+                                         RingPos &pos, uint32_t &seg_it, uint32_t *status) {
     volatile int *ab = &sh.abort_flag;
     const uint32_t idesc = umma_idesc_bf16(ncols);
-    SegIter seg(g->tiles, g->kb_total, whole, blockIdx.x, p, gridDim.x);
-    int tile, kb0, kb1;
-    while (seg.next(tile, kb0, kb1)) {
+    const SegList &L = sh.segs[kind][p];
+    for (int i = 0; i < L.n; ++i) {
+        const int kb0 = L.kb0[i], kb1 = L.kb1[i];
         const int buf = seg_it & 1;
         const uint32_t aph = (seg_it >> 1) & 1u;
         if (!mbar_wait(smem_u32(&sh.acc_empty[p][buf]), aph ^ 1u, ab, status)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tmem_d = sh.tmem + (p * 2 + buf) * kMegaAccCols;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-            const int s = it % ring.stages;
-            const uint32_t ph = (it / ring.stages) & 1u;
-            if (!mbar_wait(smem_u32(&sh.w_full[p][s]), ph, ab, status)) return false;
-            if (!mbar_wait(smem_u32(&sh.x_full[p][s]), ph, ab, status)) return false;
+        for (int kb = kb0; kb < kb1; ++kb) {
+            if (!mbar_wait(smem_u32(&sh.w_full[p][pos.s]), pos.ph, ab, status)) return false;
+            if (!mbar_wait(smem_u32(&sh.x_full[p][pos.s]), pos.ph, ab, status)) return false;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t ad = umma_desc_sw128(ring.base + s * ring.stage_bytes);
-            const uint64_t bd = umma_desc_sw128(ring.base + s * ring.stage_bytes + kWTileBytes);
+            const uint64_t ad = umma_desc_sw128(ring.base + pos.s * ring.stage_bytes);
+            const uint64_t bd = umma_desc_sw128(ring.base + pos.s * ring.stage_bytes + kWTileBytes);
 #pragma unroll
             for (int k = 0; k < kTileK / 16; ++k)
                 umma_bf16(tmem_d, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), idesc, (kb > kb0 || k) ? 1u : 0u);
-            umma_commit(smem_u32(&sh.empty[p][s]));
+            umma_commit(smem_u32(&sh.empty[p][pos.s]));
+            pos.advance(ring.stages);
         }
         umma_commit(smem_u32(&sh.acc_full[p][buf]));
         ++seg_it;
@@ -795,19 +825,19 @@ __device__ __forceinline__ void mega_acc_ld8(uint32_t taddr, int c0, int t_box, 
 }
 
 // warps 6..9, split-K projections: drain the accumulators of both pipelines' segments, alternating
-__device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, const MegaArgs &m, MegaShared &sh,
+__device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, const MegaArgs &m, MegaShared &sh,
                                                    uint32_t *seg_it, int warp, int lane) {
     volatile int *ab = &sh.abort_flag;
     const int lg = warp & 3;
-    SegIter seg0(g->tiles, g->kb_total, 0, blockIdx.x, 0, gridDim.x), seg1(g->tiles, g->kb_total, 0, blockIdx.x, 1, gridDim.x);
+    const SegList &L0 = sh.segs[kind][0], &L1 = sh.segs[kind][1];
     const size_t stride = (size_t)m.T_pad * g->N;
-    bool more0 = true, more1 = true;
-    while (more0 || more1) {
+    const int rounds = L0.n > L1.n ? L0.n : L1.n;
+    for (int i = 0; i < rounds; ++i) {
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
-            int tile, kb0, kb1;
-            bool has = p ? (more1 && (more1 = seg1.next(tile, kb0, kb1))) : (more0 && (more0 = seg0.next(tile, kb0, kb1)));
-            if (!has) continue;
+            const SegList &L = p ? L1 : L0;
+            if (i >= L.n) continue;
+            const int tile = L.tile[i];
             const int buf = seg_it[p] & 1;
             const uint32_t aph = (seg_it[p] >> 1) & 1u;
             if (!mbar_wait(smem_u32(&sh.acc_full[p][buf]), aph, ab, m.status)) return false;
@@ -822,8 +852,8 @@ __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, const Mega
                 mega_acc_ld8(taddr, c0, m.t_box, m.planes, v);
                 if (n < g->N) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (c0 + i < m.T_pad) m.part[slot * stride + (size_t)(c0 + i) * g->N + n] = v[i];
+                    for (int j = 0; j < 8; ++j)
+                        if (c0 + j < m.T_pad) m.part[slot * stride + (size_t)(c0 + j) * g->N + n] = v[j];
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -842,9 +872,9 @@ __device__ __forceinline__ bool mega_epilogue_head(const MegaGemm *g, const Mega
                                                    uint32_t *seg_it, int warp, int lane) {
     volatile int *ab = &sh.abort_flag;
     const int lg = warp & 3;
-    SegIter seg(g->tiles, g->kb_total, 1, blockIdx.x, 0, gridDim.x);
-    int tile, kb0, kb1;
-    while (seg.next(tile, kb0, kb1)) {
+    const SegList &L = sh.segs[4][0];
+    for (int si = 0; si < L.n; ++si) {
+        const int tile = L.tile[si];
         uint32_t taddr[2];
         int bufs[2];
 #pragma unroll
@@ -1009,6 +1039,7 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     mega_prep_rows(m, sh);
+    mega_fill_seglists(m, sh);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1018,18 +1049,19 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         if (lane == 0) mega_w_producer(m, warp, ring[warp], sh);
     } else {
         const int gw = (warp - 2) * gridDim.x + blockIdx.x, ngw = (kMegaWorkers / 32) * gridDim.x;
-        uint32_t it = 0, seg_it[2] = {0, 0}, pg_it = 0;   // per-thread progress counters of the role loops
+        uint32_t seg_it[2] = {0, 0}, pg_it = 0;   // per-thread progress counters of the role loops
+        RingPos pos;
         const CUtensorMap *tmX[3] = {&tmXd, &tmXo, &tmXf};
-        auto gemm_phase = [&](const MegaGemm *g, int whole, int xbuf) {
+        auto gemm_phase = [&](const MegaGemm *g, int kind, int xbuf) {
             if (warp == 2 || warp == 3) {
                 const int p = warp - 2;
-                if (lane == 0) mega_mma(g, whole, p, ncols, ring[p], sh, it, seg_it[p], m.status);
+                if (lane == 0) mega_mma(kind, p, ncols, ring[p], sh, pos, seg_it[p], m.status);
             } else if (warp == 4 || warp == 5) {
                 const int p = warp - 4;
-                if (lane == 0) mega_x_load(g, whole, p, tmX[xbuf], ring[p], sh, it, m.status);
+                if (lane == 0) mega_x_load(kind, p, tmX[xbuf], ring[p], sh, pos, m.status);
             } else {
-                if (whole) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
-                else mega_epilogue_part(g, m, sh, seg_it, warp, lane);
+                if (kind == 4) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
+                else mega_epilogue_part(g, kind, m, sh, seg_it, warp, lane);
             }
             grid_sync(m, sh);
         };
@@ -1045,19 +1077,19 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
             grid_sync(m, sh);
             ew_attn_merge<HD>(m, sh, gw, ngw, lane);
             grid_sync(m, sh);
-            gemm_phase(&G4[1], 0, 1);
+            gemm_phase(&G4[1], 1, 1);
             ew_resid(m, sh, G4[1], m.ffn_norm[l], nullptr, nullptr, gw, ngw, lane);
             grid_sync(m, sh);
-            gemm_phase(&G4[2], 0, 0);
+            gemm_phase(&G4[2], 2, 0);
             ew_silu(m, G4[2], gw, ngw, lane);
             grid_sync(m, sh);
-            gemm_phase(&G4[3], 0, 2);
+            gemm_phase(&G4[3], 3, 2);
             const bool last = l + 1 == a.l1;
             ew_resid(m, sh, G4[3], last ? m.final_norm : m.attn_norm[l + 1], last ? m.exit_buf : nullptr,
                      last ? m.hidden_out : nullptr, gw, ngw, lane);
             grid_sync(m, sh);
         }
-        gemm_phase(m.head, 1, 0);
+        gemm_phase(m.head, 4, 0);
         for (int b = blockIdx.x; b < a.batch; b += gridDim.x) mega_accept(m, sh, b);
     }
     __syncthreads();
