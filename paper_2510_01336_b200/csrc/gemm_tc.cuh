@@ -74,6 +74,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
         "l"(tm), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// weight tiles are read once: evict-first keeps them from displacing re-read data in L2
+__device__ __forceinline__ void tma_load_2d_stream(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar,
+                                                   uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+        "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
@@ -175,10 +188,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             // Weights do not depend on the previous kernel: fill the ring with weight tiles
             // first, then wait for the producer of the activations.
             int pre = nkb < g.stages ? nkb : g.stages;
+            const uint64_t policy = l2_policy_evict_first();
             for (int i = 0; i < pre; ++i) {
                 uint32_t fb = smem_u32(&bar_full[i]);
                 mbar_expect_tx(fb, stage_bytes);
-                tma_load_2d(smem0 + i * stage_bytes, &tmW, (kb0 + i) * kTileK, tile * kWeightTileRows, fb);
+                tma_load_2d_stream(smem0 + i * stage_bytes, &tmW, (kb0 + i) * kTileK, tile * kWeightTileRows, fb, policy);
             }
             pdl_wait();
             for (int i = 0; i < pre; ++i)
@@ -190,7 +204,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, abort_flag, g.status)) break;
                 uint32_t fb = smem_u32(&bar_full[s]);
                 mbar_expect_tx(fb, stage_bytes);
-                tma_load_2d(smem0 + s * stage_bytes, &tmW, (kb0 + i) * kTileK, tile * kWeightTileRows, fb);
+                tma_load_2d_stream(smem0 + s * stage_bytes, &tmW, (kb0 + i) * kTileK, tile * kWeightTileRows, fb, policy);
                 tma_load_3d(smem0 + s * stage_bytes + kWTileBytes, &tmX, (kb0 + i) * kTileK, g.row0, 0, fb);
                 if (++s == g.stages) { s = 0; ph ^= 1u; }
             }

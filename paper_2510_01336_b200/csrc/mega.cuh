@@ -756,12 +756,15 @@ __device__ __forceinline__ void mega_w_producer(const MegaArgs &m, int p, const 
     volatile int *ab = &sh.abort_flag;
     WCursor ld(&m, &sh, p);
     RingPos pos;
+    // weights are read exactly once per call: mark their lines evict-first so that they do not push the
+    // partial sums, activations and KV pages (which are re-read) out of L2
+    const uint64_t policy = l2_policy_evict_first();
     while (ld.valid) {
         if (!mbar_wait(smem_u32(&sh.empty[p][pos.s]), pos.ph ^ 1u, ab, m.status)) return;
         const uint32_t fb = smem_u32(&sh.w_full[p][pos.s]);
         mbar_expect_tx(fb, kWTileBytes);
         const MegaGemm *g = ld.gemm();
-        tma_load_2d(ring.base + pos.s * ring.stage_bytes, &g->tmW, ld.kb * kTileK, ld.tile * kWeightTileRows, fb);
+        tma_load_2d_stream(ring.base + pos.s * ring.stage_bytes, &g->tmW, ld.kb * kTileK, ld.tile * kWeightTileRows, fb, policy);
         ld.advance();
         pos.advance(ring.stages);
     }
