@@ -633,7 +633,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     // one attention item per CTA where possible: the phase is latency-bound at small batch
     m.n_splits = c->sm_count / (a.batch * d.n_kv_heads * m.n_mg);
     if (m.n_splits < 1) m.n_splits = 1;
-    if (m.n_splits > 64) m.n_splits = 64;
+    if (m.n_splits > 16) m.n_splits = 16;   // one load batch in the split merge
     if ((size_t)m.n_splits * T_pad * d.n_q_heads * (d.head_dim + 2) > c->attn_part_floats) return 1;
     m.scale_log2 = (1.0f / sqrtf((float)d.head_dim)) * 1.4426950408889634f;
     m.r.len_d = kv.len_draft; m.r.len_i = kv.len_inter; m.r.len_f = kv.len_target;

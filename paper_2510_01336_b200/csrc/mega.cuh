@@ -478,43 +478,43 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
         float inv = 0.f;
         if (j < sh.nr[b]) {
             const float *base = m.attn_part + ((size_t)t * m.hq + h) * m.n_splits * (HD + 2);
-            float ms[2], ls[2];   // splits lane and lane + 32 (n_splits <= 64)
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int sidx = lane + 32 * u;
-                ms[u] = -INFINITY; ls[u] = 0.f;
-                if (sidx < m.n_splits) {
-                    ms[u] = base[(size_t)sidx * (HD + 2) + HD];
-                    ls[u] = base[(size_t)sidx * (HD + 2) + HD + 1];
-                    if (!(ls[u] > 0.f)) { ms[u] = -INFINITY; ls[u] = 0.f; }
+            // all loads of up to 16 splits go out before anything is used: one L2 round trip per batch
+            float L = 0.f, M = -INFINITY;
+            for (int s0 = 0; s0 < m.n_splits; s0 += 16) {
+                float rv[16][E];
+                float ms = -INFINITY, ls = 0.f;   // lane u < 16 holds (max, sum) of split s0 + u
+                if (lane < 16 && s0 + lane < m.n_splits) {
+                    ms = base[(size_t)(s0 + lane) * (HD + 2) + HD];
+                    ls = base[(size_t)(s0 + lane) * (HD + 2) + HD + 1];
                 }
-            }
-            float M = fmaxf(ms[0], ms[1]);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-            float wv[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) wv[u] = (ms[u] == -INFINITY) ? 0.f : exp2f(ms[u] - M);
-            float L = 0.f;
-            for (int s0 = 0; s0 < m.n_splits; s0 += 8) {
-                float rv[8][E];   // issue the loads of eight splits before using any of them
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 16; ++u) {
                     const int sidx = s0 + u < m.n_splits ? s0 + u : m.n_splits - 1;
                     const float *r = base + (size_t)sidx * (HD + 2) + lane * E;
 #pragma unroll
                     for (int e = 0; e < E; ++e) rv[u][e] = r[e];
                 }
+                if (!(ls > 0.f)) { ms = -INFINITY; ls = 0.f; }
+                float Mb = ms;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int sidx = s0 + u;
-                    if (sidx >= m.n_splits) break;
-                    const float w = __shfl_sync(0xffffffffu, wv[sidx >> 5], sidx & 31);
-                    const float l = __shfl_sync(0xffffffffu, ls[sidx >> 5], sidx & 31);
+                for (int o = 8; o > 0; o >>= 1) Mb = fmaxf(Mb, __shfl_xor_sync(0xffffffffu, Mb, o));
+                Mb = __shfl_sync(0xffffffffu, Mb, 0);
+                const float Mn = fmaxf(M, Mb);
+                const float corr = (M == -INFINITY) ? 0.f : exp2f(M - Mn);   // rescale what earlier batches added
+                L *= corr;
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[e] *= corr;
+                const float wl = (ms == -INFINITY) ? 0.f : exp2f(ms - Mn);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    if (s0 + u >= m.n_splits) break;
+                    const float w = __shfl_sync(0xffffffffu, wl, u);
+                    const float l = __shfl_sync(0xffffffffu, ls, u);
                     L += l * w;
 #pragma unroll
                     for (int e = 0; e < E; ++e) acc[e] += w * rv[u][e];
                 }
+                M = Mn;
             }
             inv = L > 0.f ? 1.0f / L : 0.f;
         }
@@ -774,12 +774,17 @@ __device__ __forceinline__ bool mega_x_load(int kind, int p, const CUtensorMap *
                                             MegaShared &sh, RingPos &pos, uint32_t *status) {
     volatile int *ab = &sh.abort_flag;
     const SegList &L = sh.segs[kind][p];
+    uint64_t policy;   // the activation operand is re-read by every CTA: keep it in L2
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
     for (int i = 0; i < L.n; ++i) {
         for (int kb = L.kb0[i]; kb < L.kb1[i]; ++kb) {
             if (!mbar_wait(smem_u32(&sh.empty[p][pos.s]), pos.ph ^ 1u, ab, status)) return false;
             const uint32_t fb = smem_u32(&sh.x_full[p][pos.s]);
             mbar_expect_tx(fb, ring.x_bytes);
-            tma_load_3d(ring.base + pos.s * ring.stage_bytes + kWTileBytes, tmX, kb * kTileK, 0, 0, fb);
+            asm volatile(
+                "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+                ::"r"(ring.base + pos.s * ring.stage_bytes + kWTileBytes), "l"(tmX), "r"(kb * kTileK), "r"(0), "r"(0), "r"(fb),
+                "l"(policy) : "memory");
             pos.advance(ring.stages);
         }
     }
