@@ -264,6 +264,72 @@ def cpu_super_round(shape, w_gpu, budget_steps: int):
             "s_per_step": total / budget_steps}
 
 
+def run_sweep(args):
+    """Verify-step latency vs k (rows per sequence) x batch x context on the Llama-3-8B shape: one
+    hispec_verify_intermediate call over [8, L_i) + exit head from seeded random state, median of 15 calls.
+    Prints one JSON line per point (not the benchmark line)."""
+    import torch
+    from paper_2510_01336_b200 import binding, workload as wl
+    import dataclasses
+    torch.cuda.set_device(0)
+    peak, peak_kind = peaks()
+    free_b, _ = torch.cuda.mem_get_info()
+    for L_i in ([16] if not args.sweep_all_li else [12, 16, 24]):
+        shape = dataclasses.replace(wl.L3_8B, L_i=L_i)
+        layers = list(range(shape.L_d, L_i))
+        w = wl.make_weights(shape, layers=layers, device="cuda", with_emb=False)
+        for B in (1, 4, 16, 64):
+            for ctx_len in (512, 4096, 32768):
+                kv_bytes = 2 * B * (ctx_len + 32) * len(layers) * shape.kv_bytes_per_token_layer // 2 * 1
+                kv_bytes = B * (ctx_len + 32) * len(layers) * shape.kv_bytes_per_token_layer
+                if kv_bytes > 0.8 * free_b:
+                    print(json.dumps({"sweep": True, "L_i": L_i, "B": B, "ctx": ctx_len, "fits": False,
+                                      "kv_gb": kv_bytes / 1e9}), flush=True)
+                    continue
+                max_pages = (ctx_len + 32 + 15) // 16
+                ctxo = binding.Context(shape, w, page_size=16, max_batch=B, max_rows_per_seq=17, max_pages_per_seq=max_pages)
+                st = ctxo.new_state(B, B * max_pages, wl.make_block_table(shape, B, max_pages), first_layer=shape.L_d,
+                                    n_pool_layers=len(layers))
+                g = torch.Generator(device="cuda").manual_seed(shape.seed + 4000)
+                st.k_pages.normal_(generator=g)
+                st.v_pages.normal_(generator=g)
+                st.h_draft.normal_(generator=g)
+                res = ctxo.new_result(B)
+                for k in (1, 2, 4, 8, 16):
+                    kd = max(k - 1, 1)
+                    drafts = torch.zeros((B, kd), dtype=torch.int32, device="cuda")
+                    nd = torch.full((B,), k - 1, dtype=torch.int32, device="cuda")
+                    nr = torch.full((B,), k, dtype=torch.int32, device="cuda")
+                    times = []
+                    for it in range(18):
+                        st.len_draft.fill_(ctx_len + k)
+                        st.len_inter.fill_(ctx_len)
+                        st.len_target.fill_(ctx_len)
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        ctxo.verify_intermediate(st, drafts, nd, nr, res, k=k - 1 if k > 1 else 0)
+                        e1.record()
+                        torch.cuda.synchronize()
+                        if it >= 3:
+                            times.append(e0.elapsed_time(e1))
+                    times.sort()
+                    ms = times[len(times) // 2]
+                    T = B * k
+                    by = (len(layers) * shape.layer_weight_bytes + shape.head_bytes +
+                          B * len(layers) * shape.kv_bytes_per_token_layer * (ctx_len + k) + 2 * T * shape.d_model * 4)
+                    fl = 2.0 * T * (len(layers) * shape.layer_params + shape.vocab * shape.d_model) + \
+                        B * len(layers) * 4.0 * shape.n_q_heads * shape.head_dim * k * (ctx_len + (k + 1) / 2)
+                    print(json.dumps({"sweep": True, "L_i": L_i, "B": B, "ctx": ctx_len, "k": k, "us": round(ms * 1e3, 1),
+                                      "algorithmic_gb": round(by / 1e9, 3), "gbs": round(by / ms / 1e6, 0),
+                                      "frac_of_measured_hbm": round(by / ms / 1e6 / peak, 3), "tflops": round(fl / ms / 1e9, 1),
+                                      "status": ctxo.status()}), flush=True)
+                ctxo.close()
+                del st, ctxo
+                torch.cuda.empty_cache()
+        del w
+        torch.cuda.empty_cache()
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
@@ -290,11 +356,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="verify-step latency vs k / batch / context (not the bench line)")
+    ap.add_argument("--sweep-all-li", action="store_true", help="sweep intermediate exits 12, 16, 24 instead of 16 only")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)

@@ -586,6 +586,15 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     const int planes = plain ? 1 : 2;
     if (!x->mega_ok || T_pad * planes > kMegaAccCols) return 1;
     const hispec_kv &kv = *sc.kv;
+    {
+        // The persistent kernel is built for calls dominated by the weight stream.  When the KV cache
+        // a layer may have to read (by the block-table capacity; the lengths live on the device) outweighs
+        // the layer's weights, the stand-alone attention kernel with its deeper page pipeline serves better.
+        double kv_cap = (double)a.batch * d.max_pages_per_seq * d.page_size * 4.0 * d.n_kv_heads * d.head_dim;
+        double w_layer = 0.0;
+        for (int k = 0; k < G_HEAD; ++k) w_layer += 2.0 * (double)c->plan[k].N * c->plan[k].K;
+        if (kv_cap > w_layer && !env_int("HISPEC_FORCE_MEGA", 0)) return 1;
+    }
     MegaArgs m;
     memset(&m, 0, sizeof(m));
     m.a = a;
@@ -632,6 +641,10 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     m.mt = ceil_div(QR < 64 ? QR : 64, 16);
     // one attention item per CTA where possible: the phase is latency-bound at small batch
     m.n_splits = c->sm_count / (a.batch * d.n_kv_heads * m.n_mg);
+    {   // ... but long sequences still want about 64 pages per item
+        int by_len = ceil_div(d.max_pages_per_seq, 64);
+        if (m.n_splits < by_len) m.n_splits = by_len;
+    }
     if (m.n_splits < 1) m.n_splits = 1;
     if (m.n_splits > 16) m.n_splits = 16;   // one load batch in the split merge
     if ((size_t)m.n_splits * T_pad * d.n_q_heads * (d.head_dim + 2) > c->attn_part_floats) return 1;
