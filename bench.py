@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 N_PROMPT, N_D, ROUNDS = 1024, 5, 2
 # dram__bytes_read.sum + dram__bytes_write.sum of one hispec_stage_kernel launch (a verify-I call of this
 # workload: layers [8,16) + head, 6 rows, context 1024) from the ncu capture summarised under profiles/
-ROOFLINE_TRAFFIC_BYTES_PER_LAUNCH = 4.687e9
+ROOFLINE_TRAFFIC_BYTES_PER_LAUNCH = 4.627e9
 
 
 def peaks():
