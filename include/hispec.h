@@ -238,6 +238,12 @@ int hispec_exit_argmax_noalloc(void *stream, const void *head, const float *fina
                                int d_model, int vocab, const float *hidden, int n_rows, int32_t *argmax_ids,
                                float *top2);
 
+/* Debug aid: with HISPEC_TRACE=1 in the environment at hispec_create(), the persistent kernel stamps the
+ * global timer after each of its grid barriers (block 0); this synchronises the device and copies the 1024
+ * stamp slots of the last call into `out` (slot 1023 = kernel start).  Returns the number of slots copied, 0
+ * when tracing is off or cap < 1024. */
+int hispec_debug_trace(hispec_ctx *ctx, unsigned long long *out, int cap);
+
 /* Text of the most recent CUDA failure behind a HISPEC_ECUDA return (process-wide, not thread-safe). */
 const char *hispec_last_error(void);
 

@@ -27,7 +27,8 @@ ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["hispec_create", "hispec_destroy", "hispec_draft", "hispec_verify_intermediate", "hispec_verify_target",
            "hispec_prefill", "hispec_device_status", "hispec_launch_count", "hispec_strerror",
-           "hispec_profile_enable", "hispec_profile_read", "hispec_last_error", "hispec_exit_argmax_noalloc"]
+           "hispec_profile_enable", "hispec_profile_read", "hispec_last_error", "hispec_exit_argmax_noalloc",
+           "hispec_debug_trace"]
 
 
 class ModelDesc(ctypes.Structure):

@@ -131,6 +131,7 @@ struct GemmArgs {
     int kb_total, splits;
     int row0, rows;      // activation rows [row0, row0 + rows) of the call
     int t_box, planes;   // rows per plane in the B tile (multiple of 8), 1 or 2 planes
+    int split_planes;    // 2 planes with more than 128 rows: one MMA per plane (N = t_box each), lo accumulator at column 256
     int stages;
     int tmem_cols;       // power of two >= max(32, t_box * planes)
     int head;            // 0: store partial sums; 1: exit head (top-2 per column, optional logits)
@@ -156,7 +157,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int kb0 = (int)((long long)g.kb_total * sp / g.splits);
     const int kb1 = (int)((long long)g.kb_total * (sp + 1) / g.splits);
     const int nkb = kb1 - kb0;
-    const int ncols = g.t_box * g.planes;
+    const int ncols = g.t_box * g.planes;                 // rows of the B tile in shared memory
+    const int mma_n = g.split_planes ? g.t_box : ncols;   // N of one MMA
+    const int lo_col = g.split_planes ? 256 : g.t_box;    // accumulator column where the lo plane's results start
     const uint32_t x_bytes = (uint32_t)ncols * 128u;
     const uint32_t stage_bytes = kWTileBytes + x_bytes;
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -211,7 +214,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(ncols);
+            const uint32_t idesc = umma_idesc_bf16(mma_n);
             bool ok = true;
             int s = 0;
             uint32_t ph = 0;
@@ -222,8 +225,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 uint64_t ad = umma_desc_sw128(smem0 + s * stage_bytes);
                 uint64_t bd = umma_desc_sw128(smem0 + s * stage_bytes + kWTileBytes);
 #pragma unroll
-                for (int k = 0; k < kTileK / 16; ++k)
+                for (int k = 0; k < kTileK / 16; ++k) {
                     umma_bf16(tmem_d, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), idesc, (i | k) ? 1u : 0u);
+                    if (g.split_planes)   // the lo plane sits t_box rows (128 bytes each) further on in the tile
+                        umma_bf16(tmem_d + 256u, ad + (uint64_t)(2 * k), bd + (uint64_t)((g.t_box * 128) >> 4) + (uint64_t)(2 * k),
+                                  idesc, (i | k) ? 1u : 0u);
+                }
                 umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
                 if (++s == g.stages) { s = 0; ph ^= 1u; }
             }
@@ -242,7 +249,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 float v[8], w[8];
                 tmem_ld8(taddr + (uint32_t)c0, v);
                 if (g.planes == 2) {
-                    tmem_ld8(taddr + (uint32_t)(g.t_box + c0), w);
+                    tmem_ld8(taddr + (uint32_t)(lo_col + c0), w);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) v[i] += w[i];
                 }

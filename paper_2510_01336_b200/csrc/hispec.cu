@@ -510,7 +510,7 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
     const bool head = kind == G_HEAD;
     const size_t split_stride = (size_t)T_pad * p.N;
     if (!head && (size_t)p.splits * split_stride > c->part_floats) return HISPEC_ECAPACITY;
-    const int chunk = planes == 2 ? 128 : 256;
+    const int chunk = 256;   // rows one launch can take (with hi/lo planes beyond 128 rows: one MMA per plane)
     for (int row0 = 0; row0 < T_pad; row0 += chunk) {
         int rows = T_pad - row0 < chunk ? T_pad - row0 : chunk;
         ProfScope prof(c, st, 10 + (int)kind, 2.0 * (double)p.N * (double)p.K);
@@ -533,10 +533,12 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
         g.N = p.N; g.K = p.K; g.kb_total = p.kb_total; g.splits = head ? 1 : p.splits;
         g.row0 = row0; g.rows = rows;
         g.planes = planes;
-        g.t_box = round_up(rows, planes == 2 ? 8 : 16);
+        g.split_planes = (planes == 2 && rows > 128) ? 1 : 0;
+        g.t_box = round_up(rows, (planes == 2 && !g.split_planes) ? 8 : 16);
         int ncols = g.t_box * planes;
         int tc = 32;
         while (tc < ncols) tc <<= 1;
+        if (g.split_planes) tc = 512;
         g.tmem_cols = tc;
         int stage_bytes = kWTileBytes + ncols * 128;
         int stages = x->gemm_smem_budget / stage_bytes;
@@ -684,8 +686,18 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     double wbytes = 2.0 * (double)c->plan[G_HEAD].N * c->plan[G_HEAD].K;
     for (int k = 0; k < G_HEAD; ++k) wbytes += 2.0 * (double)c->plan[k].N * c->plan[k].K * (a.l1 - a.l0);
     ProfScope prof(c, st, 20, wbytes);
-    if (d.head_dim == 64) CK(cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m));
-    else CK(cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m));
+    cudaError_t le = (d.head_dim == 64)
+                         ? cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m)
+                         : cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m);
+    if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorLaunchOutOfResources) {
+        // the GPU cannot hold one CTA per SM at once (e.g. it is shared): use the kernel sequence from now on
+        (void)cudaGetLastError();
+        x->mega_ok = false;
+        x->bar_sel ^= 1;
+        c->launches--;
+        return 1;
+    }
+    CK(le);
     return HISPEC_OK;
 }
 
