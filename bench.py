@@ -211,11 +211,68 @@ def run_ours(args, rank, world, local_rank):
                      "algorithmic_bytes_per_launch": roof_bytes / max(g_n, 1), "weight_bytes_per_launch": g_wbytes / max(g_n, 1),
                      "peak_source": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0},
     }
+    if not args.no_extras and world == 1:
+        line["config"]["context_same_box"] = extras(shape, w, args)
     if not args.no_cpu_baseline and world == 1:
         del loop, ctx, st
         torch.cuda.empty_cache()
         line["cpu_baseline"] = cpu_super_round(shape, w, budget_steps=1)
     print(json.dumps(line), flush=True)
+
+
+def extras(shape, w, args):
+    """Context numbers on the same box (not the headline): plain auto-regressive decoding and Algorithm 1 on the
+    literal weights, and HiSpec / Algorithm 1 / AR on acceptance-shaped weights (Wo, Wdown of the layers above the
+    draft exit scaled by 0.05, so that the exits agree as trained early-exit checkpoints do)."""
+    import torch
+    from paper_2510_01336_b200 import binding, workload as wl
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecLoop, SelfSpecLoop
+    out = {}
+    max_rows = ROUNDS * (N_D + 1) + 1
+    max_pages = (N_PROMPT + 1024 + 15) // 16
+    prompt = wl.make_tokens(shape, N_PROMPT).tolist()
+
+    def timed_tokens(make_loop, run, weights):
+        ctx = binding.Context(shape, weights, page_size=16, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+        st = ctx.new_state(1, max_pages, wl.make_block_table(shape, 1, max_pages))
+        loop = make_loop(ctx, st)
+        loop.prefill([prompt])
+        l0 = int(st.len_target[0])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        run(loop)
+        e1.record()
+        torch.cuda.synchronize()
+        toks = int(st.len_target[0]) - l0
+        stats = getattr(loop, "stats", None)
+        ctx.close()
+        return toks / (e0.elapsed_time(e1) * 1e-3), toks, stats
+
+    def run_ar(loop):
+        loop.generate(48)
+
+    def run_hs(loop):
+        for _ in range(12):
+            loop.enqueue_super_round()
+
+    def run_ss(loop):
+        for _ in range(16):
+            loop.enqueue_round()
+
+    out["ar_tokens_per_s"] = round(timed_tokens(lambda c, s: ARLoop(c, s, 1), run_ar, w)[0], 1)
+    out["selfspec_alg1_tokens_per_s"] = round(timed_tokens(lambda c, s: SelfSpecLoop(c, s, 1, N_D), run_ss, w)[0], 1)
+    wg = wl.make_weights(shape, device="cuda", resid_scale={l: 0.05 for l in range(shape.L_d, shape.L_f)})
+    tps, toks, stats = timed_tokens(lambda c, s: HiSpecLoop(c, s, 1, N_D, ROUNDS), run_hs, wg)
+    ss = timed_tokens(lambda c, s: SelfSpecLoop(c, s, 1, N_D), run_ss, wg)
+    ar = timed_tokens(lambda c, s: ARLoop(c, s, 1), run_ar, wg)[0]
+    out["acceptance_shaped_gamma0.05"] = {"hispec_tokens_per_s": round(tps, 1), "tokens_per_super_round": round(toks / 12, 2),
+                                          "selfspec_alg1_tokens_per_s": round(ss[0], 1), "tokens_per_alg1_round": round(ss[1] / 16, 2),
+                                          "ar_tokens_per_s": round(ar, 1), "hispec_over_ar": round(tps / ar, 2),
+                                          "hispec_over_alg1": round(tps / ss[0], 2)}
+    del wg
+    torch.cuda.empty_cache()
+    return out
 
 
 def cpu_super_round(shape, w_gpu, budget_steps: int):
@@ -356,6 +413,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the AR / Algorithm 1 / acceptance-shaped context numbers")
     ap.add_argument("--sweep", action="store_true", help="verify-step latency vs k / batch / context (not the bench line)")
     ap.add_argument("--sweep-all-li", action="store_true", help="sweep intermediate exits 12, 16, 24 instead of 16 only")
     args = ap.parse_args()

@@ -130,6 +130,105 @@ class HiSpecLoop:
         return [t[:n_gen] for t in self.tokens]
 
 
+class HiSpecDynamicLoop(HiSpecLoop):
+    """Algorithm 2 with the paper's dynamic trigger (Sec. 3.4): intermediate rounds continue until at
+    least N_i tokens are tentatively accepted, then the target verifies them.  The host reads the accepted
+    count after every intermediate verification (one small device-to-host copy per round) to decide."""
+
+    def __init__(self, ctx, st, batch, N_d, N_i, device="cuda"):
+        max_rounds = (ctx.max_rows - 1) // (N_d + 1)
+        assert max_rounds >= 1 and N_i + N_d + 1 <= ctx.max_rows - 1, "hidden buffers too small for N_i + N_d + 1 rows"
+        super().__init__(ctx, st, batch, N_d, rounds=max_rounds, bonus_inter=True, device=device)
+        self.N_i = N_i
+        self.h_len = torch.zeros((2, batch), dtype=torch.int32).pin_memory()
+
+    def enqueue_super_round(self, stream=None):
+        ctx, st, N_d, B = self.ctx, self.st, self.N_d, self.B
+        S_ptr = self.S.data_ptr()
+        s = stream if stream is not None else torch.cuda.current_stream()
+        self.rounds_used = 0
+        for r in range(self.rounds):
+            for j in range(N_d):
+                if j == 0:
+                    ctx.draft(st, self.pending, S_ptr, batch=B, in_stride=1, out_stride=N_d, stream=stream)
+                else:
+                    ctx.draft(st, S_ptr + 4 * (j - 1), S_ptr + 4 * j, batch=B, in_stride=N_d, out_stride=N_d, stream=stream)
+            ctx.draft(st, S_ptr + 4 * (N_d - 1), None, batch=B, in_stride=N_d, stream=stream)
+            ctx.verify_intermediate(st, self.S, None, None, self.res_i[r], stream=stream, k=N_d)
+            self.stats.draft_steps += N_d + 1
+            self.stats.inter_calls += 1
+            self.rounds_used += 1
+            with torch.cuda.stream(s):
+                self.h_len[0].copy_(st.len_inter, non_blocking=True)
+                self.h_len[1].copy_(st.len_target, non_blocking=True)
+            s.synchronize()
+            if int((self.h_len[0] - self.h_len[1]).min()) >= self.N_i:   # every sequence has |V| >= N_i
+                break
+        ctx.verify_target(st, self.V, None, None, self.res_t, stream=stream, k=ctx.max_rows - 1)
+        self.stats.target_calls += 1
+        self.stats.super_rounds += 1
+
+    def collect(self, stream=None):
+        rounds, self.rounds = self.rounds, self.rounds_used
+        try:
+            return super().collect(stream)
+        finally:
+            self.rounds = rounds
+
+
+class SelfSpecLoop:
+    """Algorithm 1 (single-stage self-speculation): N_d (+1) draft steps at L_d, then one verification of the
+    block by the final layer -- hispec_verify_intermediate over [L_d, L_f) with the L_f exit."""
+
+    def __init__(self, ctx: binding.Context, st: binding.KVState, batch: int, N_d: int, device: str = "cuda"):
+        assert N_d + 1 <= ctx.max_rows
+        self.ctx, self.st, self.B, self.N_d = ctx, st, batch, N_d
+        i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device=device)
+        self.pending, self.S = i32(batch), i32(batch, N_d)
+        self.res = binding.Result(i32(batch), i32(batch))
+        self.res.pending = self.pending
+        self.h = torch.zeros((2, batch), dtype=torch.int32).pin_memory()
+        self.h_S = torch.zeros((batch, N_d), dtype=torch.int32).pin_memory()
+        self.tokens: List[List[int]] = [[] for _ in range(batch)]
+
+    def prefill(self, prompts: List[List[int]]):
+        B = self.B
+        mx = max(len(p) for p in prompts)
+        toks = torch.zeros((B, mx), dtype=torch.int32)
+        for b, p in enumerate(prompts):
+            toks[b, : len(p)] = torch.tensor(p, dtype=torch.int32)
+        n = torch.tensor([len(p) for p in prompts], dtype=torch.int32)
+        self.ctx.prefill(self.st, toks.cuda(), n.cuda(), self.pending)
+        torch.cuda.synchronize()
+        self.tokens = [[t] for t in self.pending.cpu().tolist()]
+
+    def enqueue_round(self, stream=None):
+        ctx, st, N_d, B = self.ctx, self.st, self.N_d, self.B
+        S_ptr = self.S.data_ptr()
+        for j in range(N_d):
+            if j == 0:
+                ctx.draft(st, self.pending, S_ptr, batch=B, in_stride=1, out_stride=N_d, stream=stream)
+            else:
+                ctx.draft(st, S_ptr + 4 * (j - 1), S_ptr + 4 * j, batch=B, in_stride=N_d, out_stride=N_d, stream=stream)
+        ctx.draft(st, S_ptr + 4 * (N_d - 1), None, batch=B, in_stride=N_d, stream=stream)
+        ctx.verify_intermediate(st, self.S, None, None, self.res, layer_end=ctx.exits.L_f, stream=stream, k=N_d)
+
+    def collect(self):
+        self.h[0].copy_(self.res.n_accepted, non_blocking=True)
+        self.h[1].copy_(self.res.next_token, non_blocking=True)
+        self.h_S.copy_(self.S, non_blocking=True)
+        torch.cuda.synchronize()
+        for b in range(self.B):
+            a, nxt = int(self.h[0, b]), int(self.h[1, b])
+            self.tokens[b] += self.h_S[b, :a].tolist() + ([nxt] if nxt >= 0 else [])
+
+    def generate(self, n_gen: int) -> List[List[int]]:
+        while min(len(t) for t in self.tokens) < n_gen:
+            self.enqueue_round()
+            self.collect()
+        return [t[:n_gen] for t in self.tokens]
+
+
 class ARLoop:
     """Vanilla auto-regressive decoding: hispec_draft over [0, L_f) with the L_f exit, one row per step."""
 

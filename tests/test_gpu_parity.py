@@ -177,6 +177,34 @@ def test_tiny_prefill_and_free_running_lossless():
     ctx.close(); ctx2.close()
 
 
+def test_tiny_dynamic_trigger_and_single_stage_loops_are_lossless():
+    """The paper's dynamic trigger (|V| >= N_i) and Algorithm 1, free-running on the GPU with weights whose
+    exits mostly agree: both must reproduce the GPU's own auto-regressive greedy output."""
+    b = _binding()
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecDynamicLoop, SelfSpecLoop
+    shape = wl.TINY
+    scale = {l: 0.05 for l in range(shape.L_d, shape.L_f)}
+    wg = wl.make_weights(shape, resid_scale=scale).to("cuda")
+    n_prompt, n_gen, N_d, N_i = 64, 48, 2, 4
+    max_rows, max_pages = 12, (n_prompt + n_gen + 40) // 16 + 1
+    prompt = wl.make_tokens(shape, n_prompt).tolist()
+    bt = wl.make_block_table(shape, 1, max_pages)
+    outs = {}
+    for name in ("ar", "dynamic", "selfspec"):
+        ctx = b.Context(shape, wg, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+        st = ctx.new_state(1, max_pages, bt)
+        loop = {"ar": lambda: ARLoop(ctx, st, 1), "dynamic": lambda: HiSpecDynamicLoop(ctx, st, 1, N_d, N_i),
+                "selfspec": lambda: SelfSpecLoop(ctx, st, 1, N_d)}[name]()
+        loop.prefill([prompt])
+        outs[name] = loop.generate(n_gen)[0]
+        assert ctx.status() == 0
+        if name == "dynamic":
+            assert loop.stats.inter_accepted > 5 and loop.stats.target_accepted > 5
+            assert loop.stats.inter_calls > loop.stats.target_calls       # several rounds per target verification
+        ctx.close()
+    assert outs["dynamic"] == outs["ar"] and outs["selfspec"] == outs["ar"]
+
+
 @pytest.mark.parametrize("flagname,B", [("tcgen05", 3), ("simt", 3), ("rowwarp-attn", 3), ("multi-kernel", 3),
                                         ("tcgen05", 20)])
 def test_batched_ragged_gqa_pages_permuted(flagname, B):
