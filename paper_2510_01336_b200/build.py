@@ -28,6 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + ".tmp.%d" % os.getpid()
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
            "-Xcompiler", "-fPIC", "-Xptxas", "-v" if verbose else "-O3", "-o", tmp]
+    cmd += os.environ.get("HISPEC_NVCC_FLAGS", "").split()   # e.g. -DHISPEC_STAMPS for a development build
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     cmd += ["-lcudart"]
     res = subprocess.run(cmd, capture_output=True, text=True)

@@ -100,7 +100,8 @@ struct hispec_ctx_ext {
     const void *mega_heads[4];
     int n_mega_heads;
     const float **d_attn_norm, **d_ffn_norm;  // device arrays of device pointers
-    float *ssq;                // [T_alloc][ceil(d / 256)] chunk sums of squares
+    float *ssq;                // [T_alloc][ceil(d / 128)] chunk sums of squares
+    float2 *rope;              // [T_alloc][head_dim / 2] (cos, sin) of this call's rows, filled by the persistent kernel
     unsigned *bar;             // grid barrier counters, used alternately by successive launches
     int bar_sel;
     unsigned long long *trace; // debug: phase time stamps of the persistent kernel (HISPEC_TRACE=1)
@@ -298,7 +299,7 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
                 if (v > worst) worst = v;
             }
         c->attn_max_splits = (int)(worst / ((size_t)d.max_batch * d.max_rows_per_seq)) + 1;
-        c->attn_part_floats = worst * d.n_q_heads * (d.head_dim + 2);
+        c->attn_part_floats = worst * d.n_q_heads * (d.head_dim + 4);   // records padded to 16 bytes by the persistent kernel
     }
     auto alloc = [&](void **p, size_t bytes) { return cudaMalloc(p, bytes ? bytes : 16) == cudaSuccess; };
     ok = true;
@@ -321,7 +322,8 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     ok = ok && alloc((void **)&c->ext.d_gemms, sizeof(MegaGemm) * (L * 4 + 4));
     ok = ok && alloc((void **)&c->ext.d_attn_norm, sizeof(float *) * L);
     ok = ok && alloc((void **)&c->ext.d_ffn_norm, sizeof(float *) * L);
-    ok = ok && alloc((void **)&c->ext.ssq, sizeof(float) * (size_t)T_alloc * ceil_div(d.d_model, kEwChunk));
+    ok = ok && alloc((void **)&c->ext.ssq, sizeof(float) * (size_t)T_alloc * ceil_div(d.d_model, kSsqChunk));
+    ok = ok && alloc((void **)&c->ext.rope, sizeof(float2) * (size_t)T_alloc * (d.head_dim / 2));
     ok = ok && alloc((void **)&c->ext.bar, 2 * sizeof(unsigned));
     if (env_int("HISPEC_TRACE", 0)) ok = ok && alloc((void **)&c->ext.trace, 1024 * sizeof(unsigned long long));
     if (!ok) { hispec_destroy(c); return HISPEC_ENOMEM; }
@@ -376,7 +378,7 @@ extern "C" int hispec_destroy(hispec_ctx *c0) {
     hispec_ctx_full *c = static_cast<hispec_ctx_full *>(c0);
     void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->attn_part, c->top_part, c->logits_ws, c->inv_freq,
                     c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status,
-                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace};
+                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace, c->ext.rope};
     for (void *p : bufs)
         if (p) cudaFree(p);
     delete[] c->wqkv; delete[] c->wo; delete[] c->wgu; delete[] c->wdown; delete[] c->attn_norm; delete[] c->ffn_norm;
@@ -636,7 +638,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     m.k_pages = (__nv_bfloat16 *)kv.k_pages; m.v_pages = (__nv_bfloat16 *)kv.v_pages;
     m.block_table = kv.block_table; m.n_pages = kv.n_pages; m.first_layer = kv.first_layer;
     m.x = c->x; m.act_d = c->act_d; m.act_o = c->act_o; m.act_f = c->act_f; m.q = c->q; m.part = c->part;
-    m.attn_part = c->attn_part; m.top_part = c->top_part; m.ssq = x->ssq; m.inv_freq = c->inv_freq;
+    m.attn_part = c->attn_part; m.top_part = c->top_part; m.ssq = x->ssq; m.inv_freq = c->inv_freq; m.rope = x->rope;
     m.G = d.n_q_heads / d.n_kv_heads;
     const int QR = m.G * a.R_pad;
     m.n_mg = ceil_div(QR, 64);
@@ -649,7 +651,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     }
     if (m.n_splits < 1) m.n_splits = 1;
     if (m.n_splits > 16) m.n_splits = 16;   // one load batch in the split merge
-    if ((size_t)m.n_splits * T_pad * d.n_q_heads * (d.head_dim + 2) > c->attn_part_floats) return 1;
+    if ((size_t)m.n_splits * T_pad * d.n_q_heads * (d.head_dim + kAttnRecPad) > c->attn_part_floats) return 1;
     m.scale_log2 = (1.0f / sqrtf((float)d.head_dim)) * 1.4426950408889634f;
     m.r.len_d = kv.len_draft; m.r.len_i = kv.len_inter; m.r.len_f = kv.len_target;
     m.r.draft_tokens = sc.draft_tokens; m.r.token_stride = sc.token_stride; m.r.out_stride = sc.out_stride;

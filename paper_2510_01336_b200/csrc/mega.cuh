@@ -29,6 +29,7 @@
 // wait -- mbarrier or grid barrier -- is bounded; on a timeout the CTA raises an abort flag,
 // sets HISPEC_ST_TIMEOUT, and all later waits fall through so that the kernel drains and exits.
 #pragma once
+#include <type_traits>
 
 #include "attention.cuh"
 #include "gemm_tc.cuh"
@@ -42,6 +43,7 @@ constexpr int kMegaWorkers = 256;  // threads of warps 2..9
 constexpr int kMegaLeader = 64;    // warp 2 lane 0
 constexpr int kMegaAccCols = 128;  // TMEM columns per accumulator buffer (2 pipelines x 2 buffers)
 constexpr int kEwChunk = 256;      // columns per element-wise work item (one warp, 8 per lane)
+constexpr int kSsqChunk = 128;     // columns per sum-of-squares record
 
 struct __align__(64) MegaGemm {
     CUtensorMap tmW;
@@ -72,6 +74,7 @@ struct MegaArgs {
     __nv_bfloat16 *act_d, *act_o, *act_f;
     float *q, *part, *attn_part, *top_part, *ssq;
     const double *inv_freq;
+    float2 *rope;            // [T_pad][hd / 2] (cos, sin) of each row's position, filled in the first phase
     int n_splits, n_mg, mt, G;
     float scale_log2;
     AcceptArgs r;
@@ -102,10 +105,31 @@ struct MegaShared {
     int abort_flag;
     int trace_n;
     int bar_k;
+    int stamp_on, stamp_n;   // HISPEC_STAMPS builds only: fine-grained time stamps of one layer
     int p0[kMegaMaxBatch], nr[kMegaMaxBatch], nd[kMegaMaxBatch], dst[kMegaMaxBatch];
     float red_v1[8], red_v2[8];
     int red_i1[8];
 };
+
+// Development aid (compiled with -DHISPEC_STAMPS only): lane 0 of any warp of one CTA records
+// (tag * 100 + warp, global timer) pairs into the trace buffer, words 200.., while sh.stamp_on is set.
+#ifdef HISPEC_STAMPS
+#ifndef HISPEC_STAMP_CTA
+#define HISPEC_STAMP_CTA 0
+#endif
+#define MEGA_STAMP(tag)                                                                                   \
+    do {                                                                                                  \
+        if (m.trace && blockIdx.x == HISPEC_STAMP_CTA && (threadIdx.x & 31) == 0 &&                       \
+            *((volatile int *)&sh.stamp_on)) {                                                            \
+            unsigned long long t_;                                                                        \
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                         \
+            const int i_ = atomicAdd(&sh.stamp_n, 1);                                                     \
+            if (i_ < 200) { m.trace[200 + 2 * i_] = (tag) * 100 + (threadIdx.x >> 5); m.trace[201 + 2 * i_] = t_; } \
+        }                                                                                                 \
+    } while (0)
+#else
+#define MEGA_STAMP(tag) do { } while (0)
+#endif
 
 // ---- stream-K partition ----------------------------------------------------------------------
 // The k-blocks of a projection, numbered tile-major, are cut into gridDim.x equal spans.
@@ -169,13 +193,15 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
 // All worker threads of all CTAs.  Global writes made before it are visible after it, also to TMA
 // reads.  The counter only grows during a launch: barrier number k is passed once it has reached
 // (k + 1) * gridDim.x.  Arrival is a fire-and-forget release reduction; waiting polls with acquire loads.
-__device__ __forceinline__ void grid_sync(const MegaArgs &m, MegaShared &sh) {
-    asm volatile("fence.proxy.async;" ::: "memory");
+// `to_tma`: the phase wrote something that a later TMA load reads (activation planes, K/V pages).
+__device__ __forceinline__ void grid_sync(const MegaArgs &m, MegaShared &sh, bool to_tma = true) {
+    if (to_tma) asm volatile("fence.proxy.async;" ::: "memory");
     worker_bar();
     if (threadIdx.x == kMegaLeader) {
         volatile int *ab = &sh.abort_flag;
         const unsigned target = (unsigned)(++sh.bar_k) * gridDim.x;
         if (!*ab) {
+            MEGA_STAMP(60);
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(m.bar_count) : "memory");
             bool ok = false;
             for (uint32_t it = 0; it < (1u << 26); ++it) {
@@ -187,6 +213,7 @@ __device__ __forceinline__ void grid_sync(const MegaArgs &m, MegaShared &sh) {
                 atomicOr(m.status, HISPEC_ST_TIMEOUT);
             }
         }
+        MEGA_STAMP(61);
         if (m.trace && blockIdx.x == 0) {
             unsigned long long t;
             asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -245,7 +272,7 @@ __device__ __forceinline__ void mega_prep_rows(const MegaArgs &m, MegaShared &sh
 
 // 1 / rms of row t from the per-chunk sums of squares of the phase that produced the row
 __device__ __forceinline__ float mega_inv_rms(const MegaArgs &m, int t) {
-    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
+    const int nch = (m.d + kSsqChunk - 1) / kSsqChunk;
     float s = 0.f;
     for (int c = 0; c < nch; ++c) s += m.ssq[(size_t)t * nch + c];
     return rsqrtf(s / (float)m.d + m.eps);
@@ -267,18 +294,34 @@ __device__ __forceinline__ void store8_hilo(__nv_bfloat16 *hi, __nv_bfloat16 *lo
 }
 
 // sum of the split-K partial slots of 8 consecutive columns (all inside one tile), slot order
-__device__ __forceinline__ void sum_slots8(const MegaArgs &m, const MegaGemm &g, int t, int n, float *v) {
+// part 0 / 1 of `parts` = 2 takes the first ceil(ns / 2) / the remaining slots (parts = 1: all of them)
+__device__ __forceinline__ void sum_slots8(const MegaArgs &m, const MegaGemm &g, int t, int n, float *v, int part = 0,
+                                           int parts = 1) {
     int first, ns;
     mega_slots(n / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
     const size_t stride = (size_t)m.T_pad * g.N;
     const float *p = m.part + (size_t)t * g.N + n;
+    if (parts == 2) {
+        const int h0 = (ns + 1) >> 1;
+        if (part) { p += (size_t)h0 * stride; ns -= h0; } else ns = h0;
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = 0.f;
-    for (int s = 0; s < ns; ++s) {
-        float4 a = *reinterpret_cast<const float4 *>(p + s * stride);
-        float4 b = *reinterpret_cast<const float4 *>(p + s * stride + 4);
-        v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
-        v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+    // eight slots per batch, all loads in flight together; the sum stays in slot order
+    for (int s0 = 0; s0 < ns; s0 += 8) {
+        float4 a[8], b[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int sidx = s0 + u < ns ? s0 + u : ns - 1;
+            a[u] = *reinterpret_cast<const float4 *>(p + sidx * stride);
+            b[u] = *reinterpret_cast<const float4 *>(p + sidx * stride + 4);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (s0 + u < ns) {
+                v[0] += a[u].x; v[1] += a[u].y; v[2] += a[u].z; v[3] += a[u].w;
+                v[4] += b[u].x; v[5] += b[u].y; v[6] += b[u].z; v[7] += b[u].w;
+            }
     }
 }
 __device__ __forceinline__ float sum_slots1(const MegaArgs &m, const MegaGemm &g, int t, int n) {
@@ -333,58 +376,95 @@ __device__ void ew_rows_in(const MegaArgs &m, MegaShared &sh, const float *gain,
             for (int i = 0; i < 8; ++i) { ss += v[i] * v[i]; gv[i] = v[i] * gain[c + i]; }
             store8_hilo(m.act_d + (size_t)t * m.d + c, m.act_d + ((size_t)m.T_alloc + t) * m.d + c, gv, m.plain);
         }
-        ss = warp_sum(ss);
-        if (lane == 0) m.ssq[(size_t)t * nch + ch] = ss;
+        // lanes 0-15 hold the chunk's first 128 columns, lanes 16-31 the second 128: one record each
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        const int nrec = (m.d + kSsqChunk - 1) / kSsqChunk, rec = 2 * ch + (lane >> 4);
+        if ((lane & 15) == 0 && rec < nrec) m.ssq[(size_t)t * nrec + rec] = ss;
+    }
+}
+
+// (cos, sin) of every row's rotary angles, once per call (the angle is formed and reduced in fp64).
+// Dealt to the grid's worker warps from the far end, so that it runs beside ew_rows_in's items.
+__device__ void ew_rope_table(const MegaArgs &m, MegaShared &sh, int gw, int ngw, int lane) {
+    const StageArgs &a = m.a;
+    const int half = m.hd / 2;
+    for (int idx = (ngw - 1 - gw) * 32 + lane; idx < m.T_pad * half; idx += ngw * 32) {
+        const int t = idx / half, i = idx - t * half, b = t / a.R_pad, j = t - b * a.R_pad;
+        double sn, cs;
+        sincos((double)(sh.p0[b] + j) * m.inv_freq[i], &sn, &cs);
+        m.rope[idx] = make_float2((float)cs, (float)sn);
     }
 }
 
 // a5/a7 epilogue: x += projection; act_d <- hi/lo(x .* gain); chunk sums of squares; exit rows on the last layer
 __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, const float *gain, float *exit_buf,
                          float *hidden_out, int gw, int ngw, int lane) {
+    // One warp per (row, 128 columns): the half-warps each add half of the partial slots (a tile of O or
+    // down has about ten), 8 columns per lane, and exchange their sums; then half 0 stores the fp32 row,
+    // half 1 the bf16 operand planes.
     const StageArgs &a = m.a;
-    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
+    const int nch = (m.d + kSsqChunk - 1) / kSsqChunk;
+    const int hl = lane >> 4, li = lane & 15;
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
         const int t = item / nch, ch = item % nch, b = t / a.R_pad, j = t % a.R_pad;
-        const int c = ch * kEwChunk + lane * 8;
+        const int c = ch * kSsqChunk + li * 8;
         const bool valid = j < sh.nr[b];
         float ss = 0.f;
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        float4 p = make_float4(0.f, 0.f, 0.f, 0.f), q = p;
         if (c < m.d) {
-            float v[8];
-            sum_slots8(m, g, t, c, v);
-            float *xr = m.x + (size_t)t * m.d + c;
-            float4 p = *reinterpret_cast<const float4 *>(xr), q = *reinterpret_cast<const float4 *>(xr + 4);
+            const float *xr = m.x + (size_t)t * m.d + c;
+            p = *reinterpret_cast<const float4 *>(xr);
+            q = *reinterpret_cast<const float4 *>(xr + 4);
+            sum_slots8(m, g, t, c, v, hl, 2);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float o = __shfl_xor_sync(0xffffffffu, v[i], 16);
+            v[i] = hl ? o + v[i] : v[i] + o;   // first half + second half, the same value in both half-warps
+        }
+        if (c < m.d) {
             const float xo[8] = {p.x, p.y, p.z, p.w, q.x, q.y, q.z, q.w};
-            float gv[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 v[i] = valid ? v[i] + xo[i] : 0.f;
                 ss += v[i] * v[i];
-                gv[i] = v[i] * gain[c + i];
             }
-            *reinterpret_cast<float4 *>(xr) = make_float4(v[0], v[1], v[2], v[3]);
-            *reinterpret_cast<float4 *>(xr + 4) = make_float4(v[4], v[5], v[6], v[7]);
-            if (valid && exit_buf) {
-                float *e = exit_buf + ((size_t)b * a.max_rows + sh.dst[b] + j) * m.d + c;
-                *reinterpret_cast<float4 *>(e) = make_float4(v[0], v[1], v[2], v[3]);
-                *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            if (hl == 0) {
+                float *xr = m.x + (size_t)t * m.d + c;
+                *reinterpret_cast<float4 *>(xr) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4 *>(xr + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                if (valid && exit_buf) {
+                    float *e = exit_buf + ((size_t)b * a.max_rows + sh.dst[b] + j) * m.d + c;
+                    *reinterpret_cast<float4 *>(e) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                }
+                if (valid && hidden_out) {
+                    float *e = hidden_out + ((size_t)b * a.max_rows + j) * m.d + c;
+                    *reinterpret_cast<float4 *>(e) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                }
+            } else {
+                float gv[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) gv[i] = v[i] * gain[c + i];
+                store8_hilo(m.act_d + (size_t)t * m.d + c, m.act_d + ((size_t)m.T_alloc + t) * m.d + c, gv, m.plain);
             }
-            if (valid && hidden_out) {
-                float *e = hidden_out + ((size_t)b * a.max_rows + j) * m.d + c;
-                *reinterpret_cast<float4 *>(e) = make_float4(v[0], v[1], v[2], v[3]);
-                *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
-            }
-            store8_hilo(m.act_d + (size_t)t * m.d + c, m.act_d + ((size_t)m.T_alloc + t) * m.d + c, gv, m.plain);
         }
-        ss = warp_sum(ss);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if (lane == 0) m.ssq[(size_t)t * nch + ch] = ss;
     }
 }
 
-// 1 / rms of row t, lanes fetching the chunk sums in parallel (nch <= 32); same value in every lane
+// 1 / rms of row t, lanes fetching the chunk sums in parallel; same value in every lane
 __device__ __forceinline__ float mega_inv_rms_warp(const MegaArgs &m, int t, int lane) {
-    const int nch = (m.d + kEwChunk - 1) / kEwChunk;
-    if (nch > 32) return mega_inv_rms(m, t);
-    float s = lane < nch ? m.ssq[(size_t)t * nch + lane] : 0.f;
+    const int nch = (m.d + kSsqChunk - 1) / kSsqChunk;
+    float s = 0.f;
+    for (int c = lane; c < nch; c += 32) s += m.ssq[(size_t)t * nch + c];
     s = warp_sum(s);
     return rsqrtf(s / (float)m.d + m.eps);
 }
@@ -414,12 +494,24 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         const float *pr = m.part + (size_t)t * g.N + h * hd;
         if (h < m.hq + m.hkv) {
             for (int i = lane; i < half; i += 32) {
+                const float2 cs = m.rope[(size_t)t * half + i];
                 float x0 = 0.f, x1 = 0.f;
-                for (int s = 0; s < ns; ++s) { x0 += pr[s * stride + i]; x1 += pr[s * stride + i + half]; }
+                // slots eight at a time: all sixteen loads of a batch are in flight together; slots past the
+                // last one re-read it with weight zero, so the order of the sum is the slot order
+                for (int s0 = 0; s0 < ns; s0 += 8) {
+                    float u0[8], u1[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int sidx = s0 + u < ns ? s0 + u : ns - 1;
+                        u0[u] = pr[sidx * stride + i];
+                        u1[u] = pr[sidx * stride + i + half];
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (s0 + u < ns) { x0 += u0[u]; x1 += u1[u]; }
+                }
                 x0 *= inv; x1 *= inv;
-                double sn, cs;
-                sincos((double)pos * m.inv_freq[i], &sn, &cs);
-                const float c = (float)cs, sf = (float)sn;
+                const float c = cs.x, sf = cs.y;
                 const float r0 = x0 * c - x1 * sf, r1 = x1 * c + x0 * sf;
                 if (h < m.hq) {
                     m.q[(size_t)t * nq + h * hd + i] = r0;
@@ -433,10 +525,23 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         } else if (page_ok) {
             const int vh = h - m.hq - m.hkv;
             const size_t o = page_base + ((size_t)vh * a.page_size + slot) * hd;
-            for (int i = lane; i < hd; i += 32) {
-                float v = 0.f;
-                for (int s = 0; s < ns; ++s) v += pr[s * stride + i];
-                m.v_pages[o + i] = __float2bfloat16_rn(inv * v);
+            for (int i = lane; i < hd; i += 64) {
+                float v0 = 0.f, v1 = 0.f;
+                const int i1 = i + 32 < hd ? i + 32 : i;
+                for (int s0 = 0; s0 < ns; s0 += 8) {
+                    float u0[8], u1[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int sidx = s0 + u < ns ? s0 + u : ns - 1;
+                        u0[u] = pr[sidx * stride + i];
+                        u1[u] = pr[sidx * stride + i1];
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (s0 + u < ns) { v0 += u0[u]; v1 += u1[u]; }
+                }
+                m.v_pages[o + i] = __float2bfloat16_rn(inv * v0);
+                if (i + 32 < hd) m.v_pages[o + i + 32] = __float2bfloat16_rn(inv * v1);
             }
         }
     }
@@ -463,13 +568,16 @@ __device__ void ew_silu(const MegaArgs &m, const MegaGemm &g, int gw, int ngw, i
 }
 
 // a4 (second half): combine the key splits of every (row, q head) in split order -> act_o hi/lo.
-// One warp per (row, head): lanes first fetch the splits' (max, sum) pairs in parallel, then walk the
-// splits in order with the weights broadcast by shuffle, so no load waits on a branch.
+// One warp per (row, head), a lane per HD/32 columns.  Records are HD + 4 floats apart (16-byte aligned:
+// one vector load per lane and split); the (max, sum) pairs of up to 32 splits are fetched one per lane,
+// and the splits are walked in order with the weights broadcast by shuffle.
+constexpr int kAttnRecPad = 4;
 template <int HD>
 __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw, int lane) {
-    constexpr int E = HD / 32;
+    constexpr int E = HD / 32, REC = HD + kAttnRecPad;
     const StageArgs &a = m.a;
     const int nq = m.hq * HD;
+    MEGA_STAMP(30);
     for (int item = gw; item < m.T_pad * m.hq; item += ngw) {
         const int t = item / m.hq, h = item % m.hq, b = t / a.R_pad, j = t % a.R_pad;
         float acc[E];
@@ -477,42 +585,41 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
         float inv = 0.f;
         if (j < sh.nr[b]) {
-            const float *base = m.attn_part + ((size_t)t * m.hq + h) * m.n_splits * (HD + 2);
-            // all loads of up to 16 splits go out before anything is used: one L2 round trip per batch
+            const float *base = m.attn_part + ((size_t)t * m.hq + h) * m.n_splits * REC;
             float L = 0.f, M = -INFINITY;
-            for (int s0 = 0; s0 < m.n_splits; s0 += 16) {
-                float rv[16][E];
-                float ms = -INFINITY, ls = 0.f;   // lane u < 16 holds (max, sum) of split s0 + u
-                if (lane < 16 && s0 + lane < m.n_splits) {
-                    ms = base[(size_t)(s0 + lane) * (HD + 2) + HD];
-                    ls = base[(size_t)(s0 + lane) * (HD + 2) + HD + 1];
-                }
-#pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    const int sidx = s0 + u < m.n_splits ? s0 + u : m.n_splits - 1;
-                    const float *r = base + (size_t)sidx * (HD + 2) + lane * E;
-#pragma unroll
-                    for (int e = 0; e < E; ++e) rv[u][e] = r[e];
+            for (int s0 = 0; s0 < m.n_splits; s0 += 32) {
+                const int cnt = min(32, m.n_splits - s0);
+                float ms = -INFINITY, ls = 0.f;   // lane u holds (max, sum) of split s0 + u
+                if (lane < cnt) {
+                    const float2 ml = *reinterpret_cast<const float2 *>(base + (size_t)(s0 + lane) * REC + HD);
+                    ms = ml.x; ls = ml.y;
                 }
                 if (!(ls > 0.f)) { ms = -INFINITY; ls = 0.f; }
                 float Mb = ms;
 #pragma unroll
-                for (int o = 8; o > 0; o >>= 1) Mb = fmaxf(Mb, __shfl_xor_sync(0xffffffffu, Mb, o));
-                Mb = __shfl_sync(0xffffffffu, Mb, 0);
+                for (int o = 16; o > 0; o >>= 1) Mb = fmaxf(Mb, __shfl_xor_sync(0xffffffffu, Mb, o));
                 const float Mn = fmaxf(M, Mb);
                 const float corr = (M == -INFINITY) ? 0.f : exp2f(M - Mn);   // rescale what earlier batches added
                 L *= corr;
 #pragma unroll
                 for (int e = 0; e < E; ++e) acc[e] *= corr;
                 const float wl = (ms == -INFINITY) ? 0.f : exp2f(ms - Mn);
-#pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    if (s0 + u >= m.n_splits) break;
+                const float *r = base + (size_t)s0 * REC + lane * E;
+#pragma unroll 8
+                for (int u = 0; u < cnt; ++u) {
+                    float rv[E];
+                    if constexpr (E == 4) {
+                        const float4 q4 = *reinterpret_cast<const float4 *>(r + (size_t)u * REC);
+                        rv[0] = q4.x; rv[1] = q4.y; rv[2] = q4.z; rv[3] = q4.w;
+                    } else {
+                        const float2 q2 = *reinterpret_cast<const float2 *>(r + (size_t)u * REC);
+                        rv[0] = q2.x; rv[1] = q2.y;
+                    }
                     const float w = __shfl_sync(0xffffffffu, wl, u);
                     const float l = __shfl_sync(0xffffffffu, ls, u);
                     L += l * w;
 #pragma unroll
-                    for (int e = 0; e < E; ++e) acc[e] += w * rv[u][e];
+                    for (int e = 0; e < E; ++e) acc[e] += w * rv[e];
                 }
                 M = Mn;
             }
@@ -522,7 +629,9 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
         __nv_bfloat16 *olo = m.act_o + ((size_t)m.T_alloc + t) * nq + h * HD + lane * E;
 #pragma unroll
         for (int e = 0; e < E; ++e) split_hi_lo(acc[e] * inv, ohi[e], olo[e], m.plain);
+        MEGA_STAMP(31);
     }
+    MEGA_STAMP(32);
 }
 
 // ---- attention phase: items (split, kv head x row group, sequence) dealt round-robin to CTAs -------
@@ -546,6 +655,7 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
         const int pg0 = split * chunk, pg1 = min(pg0 + chunk, total_pages);
         const int n_pg = (nr > 0 && pg1 > pg0) ? pg1 - pg0 : 0;
         if (warp == 5) {
+            MEGA_STAMP(10);
             for (int i0 = 0; i0 < n_pg; i0 += 32) {
                 const int my = i0 + lane;
                 long long pgid = 0;
@@ -570,7 +680,9 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                     }
                 }
             }
+            MEGA_STAMP(12);
         } else if (warp >= 6) {
+            MEGA_STAMP(20);
             const int cw = warp - 6;
             const int r_lo = mg * 64 + cw * 16 + (lane >> 2), r_hi = r_lo + 8;
             const int j_lo = r_lo / m.G, g_lo = r_lo % m.G, j_hi = r_hi / m.G, g_hi = r_hi % m.G;
@@ -602,12 +714,14 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
             bool ok = true;
             const bool active = cw < m.mt;   // warps without rows only keep the page ring moving
+            MEGA_STAMP(21);
             for (int i = 0; i < n_pg && ok; ++i) {
                 const uint32_t it = pg_it + i;
                 const int s = it % kAttnStages;
                 const uint32_t ph = (it / kAttnStages) & 1u;
                 ok = a_wait(a_smem_u32(&sh.a_full[s]), ph, abort_flag, m.status);
                 if (!ok) break;
+                MEGA_STAMP(22);
                 if (active) {
                     const uint32_t sk = sm_attn + s * 2 * TILE, sv = sk + TILE;
                     float sc[2][4];
@@ -670,23 +784,25 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                 if (lane == 0)
                     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(&sh.a_empty[s])) : "memory");
             }
+            MEGA_STAMP(23);
             l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
             l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
             l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
             l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
             if (!ok) { l_lo = l_hi = 0.f; m_lo = m_hi = -INFINITY; }
             if (v_lo) {
-                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_lo) * m.hq + kvh * m.G + g_lo) * m.n_splits + split) * (HD + 2));
+                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_lo) * m.hq + kvh * m.G + g_lo) * m.n_splits + split) * (HD + kAttnRecPad));
 #pragma unroll
                 for (int n = 0; n < NT; ++n) *reinterpret_cast<float2 *>(dst + n * 8 + c2) = make_float2(o[n][0], o[n][1]);
                 if ((lane & 3) == 0) { dst[HD] = m_lo; dst[HD + 1] = l_lo; }
             }
             if (v_hi) {
-                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_hi) * m.hq + kvh * m.G + g_hi) * m.n_splits + split) * (HD + 2));
+                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_hi) * m.hq + kvh * m.G + g_hi) * m.n_splits + split) * (HD + kAttnRecPad));
 #pragma unroll
                 for (int n = 0; n < NT; ++n) *reinterpret_cast<float2 *>(dst + n * 8 + c2) = make_float2(o[n][2], o[n][3]);
                 if ((lane & 3) == 0) { dst[HD] = m_hi; dst[HD + 1] = l_hi; }
             }
+            MEGA_STAMP(24);
         }
         pg_it += n_pg;
     }
@@ -791,7 +907,7 @@ __device__ __forceinline__ bool mega_x_load(int kind, int p, const CUtensorMap *
     return true;
 }
 
-__device__ __forceinline__ bool mega_mma(int kind, int p, int ncols, const MegaRing &ring, MegaShared &sh,
+__device__ __forceinline__ bool mega_mma(const MegaArgs &m, int kind, int p, int ncols, const MegaRing &ring, MegaShared &sh,
                                          RingPos &pos, uint32_t &seg_it, uint32_t *status) {
     volatile int *ab = &sh.abort_flag;
     const uint32_t idesc = umma_idesc_bf16(ncols);
@@ -806,6 +922,7 @@ __device__ __forceinline__ bool mega_mma(int kind, int p, int ncols, const MegaR
         for (int kb = kb0; kb < kb1; ++kb) {
             if (!mbar_wait(smem_u32(&sh.w_full[p][pos.s]), pos.ph, ab, status)) return false;
             if (!mbar_wait(smem_u32(&sh.x_full[p][pos.s]), pos.ph, ab, status)) return false;
+            if (i == 0 && kb == kb0) MEGA_STAMP(43);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t ad = umma_desc_sw128(ring.base + pos.s * ring.stage_bytes);
             const uint64_t bd = umma_desc_sw128(ring.base + pos.s * ring.stage_bytes + kWTileBytes);
@@ -849,6 +966,7 @@ __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, 
             const int buf = seg_it[p] & 1;
             const uint32_t aph = (seg_it[p] >> 1) & 1u;
             if (!mbar_wait(smem_u32(&sh.acc_full[p][buf]), aph, ab, m.status)) return false;
+            MEGA_STAMP(45);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = sh.tmem + (p * 2 + buf) * kMegaAccCols + ((uint32_t)(lg * 32) << 16);
             const int n = tile * kWeightTileRows + lg * 32 + lane;
@@ -858,12 +976,14 @@ __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, 
             for (int c0 = 0; c0 < m.T_pad; c0 += 8) {
                 float v[8];
                 mega_acc_ld8(taddr, c0, m.t_box, m.planes, v);
+                if (c0 == 0) MEGA_STAMP(46);
                 if (n < g->N) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         if (c0 + j < m.T_pad) m.part[slot * stride + (size_t)(c0 + j) * g->N + n] = v[j];
                 }
             }
+            MEGA_STAMP(47);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0)
@@ -1019,6 +1139,8 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         sh.abort_flag = 0;
         sh.trace_n = 0;
         sh.bar_k = 0;
+        sh.stamp_on = 0;
+        sh.stamp_n = 0;
         if (blockIdx.x == 0) *((volatile unsigned *)m.bar_next) = 0u;
         if (m.trace && blockIdx.x == 0) {
             unsigned long long t;
@@ -1060,44 +1182,58 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         uint32_t seg_it[2] = {0, 0}, pg_it = 0;   // per-thread progress counters of the role loops
         RingPos pos;
         const CUtensorMap *tmX[3] = {&tmXd, &tmXo, &tmXf};
-        auto gemm_phase = [&](const MegaGemm *g, int kind, int xbuf) {
+        // `head` is a compile-time tag: the layer loop holds ONE copy of the projection roles for its four
+        // projections (a copy per projection made a layer's code larger than the instruction cache)
+        auto gemm_phase = [&](const MegaGemm *g, int kind, int xbuf, auto head) {
+            MEGA_STAMP(40 + kind);
             if (warp == 2 || warp == 3) {
                 const int p = warp - 2;
-                if (lane == 0) mega_mma(kind, p, ncols, ring[p], sh, pos, seg_it[p], m.status);
+                if (lane == 0) mega_mma(m, kind, p, ncols, ring[p], sh, pos, seg_it[p], m.status);
             } else if (warp == 4 || warp == 5) {
                 const int p = warp - 4;
                 if (lane == 0) mega_x_load(kind, p, tmX[xbuf], ring[p], sh, pos, m.status);
             } else {
-                if (kind == 4) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
+                if constexpr (decltype(head)::value) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
                 else mega_epilogue_part(g, kind, m, sh, seg_it, warp, lane);
             }
-            grid_sync(m, sh);
+            MEGA_STAMP(50 + kind);
+            grid_sync(m, sh, false);   // partial sums / top-2 records: read by plain loads
         };
         ew_rows_in(m, sh, m.attn_norm[a.l0], gw, ngw, lane);
+        ew_rope_table(m, sh, gw, ngw, lane);
         grid_sync(m, sh);
         for (int l = a.l0; l < a.l1; ++l) {
             const MegaGemm *G4 = &m.gemms[l * 4];
             const int pool_layer = l - m.first_layer;
-            gemm_phase(&G4[0], 0, 0);
-            ew_qkv(m, sh, G4[0], pool_layer, gw, ngw, lane);
-            grid_sync(m, sh);
-            mega_attention<HD>(&tmK, &tmV, m, sh, sm_attn, pool_layer, pg_it, warp, lane);
-            grid_sync(m, sh);
-            ew_attn_merge<HD>(m, sh, gw, ngw, lane);
-            grid_sync(m, sh);
-            gemm_phase(&G4[1], 1, 1);
-            ew_resid(m, sh, G4[1], m.ffn_norm[l], nullptr, nullptr, gw, ngw, lane);
-            grid_sync(m, sh);
-            gemm_phase(&G4[2], 2, 0);
-            ew_silu(m, G4[2], gw, ngw, lane);
-            grid_sync(m, sh);
-            gemm_phase(&G4[3], 3, 2);
-            const bool last = l + 1 == a.l1;
-            ew_resid(m, sh, G4[3], last ? m.final_norm : m.attn_norm[l + 1], last ? m.exit_buf : nullptr,
-                     last ? m.hidden_out : nullptr, gw, ngw, lane);
-            grid_sync(m, sh);
+#ifdef HISPEC_STAMPS
+            if (threadIdx.x == kMegaLeader) sh.stamp_on = (l == a.l0 + 3);
+#endif
+#pragma unroll 1
+            for (int kind = 0; kind < 4; ++kind) {
+                gemm_phase(&G4[kind], kind, kind == 1 ? 1 : (kind == 3 ? 2 : 0), std::false_type{});
+                if (kind == 0) {
+                    MEGA_STAMP(70);
+                    ew_qkv(m, sh, G4[0], pool_layer, gw, ngw, lane);
+                    MEGA_STAMP(71);
+                    grid_sync(m, sh);
+                    mega_attention<HD>(&tmK, &tmV, m, sh, sm_attn, pool_layer, pg_it, warp, lane);
+                    grid_sync(m, sh, false);
+                    ew_attn_merge<HD>(m, sh, gw, ngw, lane);
+                } else if (kind == 2) {
+                    MEGA_STAMP(74);
+                    ew_silu(m, G4[2], gw, ngw, lane);
+                    MEGA_STAMP(75);
+                } else {
+                    const bool last = kind == 3 && l + 1 == a.l1;
+                    const float *gain = kind == 1 ? m.ffn_norm[l] : (last ? m.final_norm : m.attn_norm[l + 1]);
+                    MEGA_STAMP(72);
+                    ew_resid(m, sh, G4[kind], gain, last ? m.exit_buf : nullptr, last ? m.hidden_out : nullptr, gw, ngw, lane);
+                    MEGA_STAMP(73);
+                }
+                grid_sync(m, sh);
+            }
         }
-        gemm_phase(m.head, 4, 0);
+        gemm_phase(m.head, 4, 0, std::true_type{});
         for (int b = blockIdx.x; b < a.batch; b += gridDim.x) mega_accept(m, sh, b);
     }
     __syncthreads();
