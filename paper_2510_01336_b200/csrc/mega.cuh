@@ -9,16 +9,16 @@
 // phases).  The other warps work phase by phase:
 //
 //   projection phase   two independent pipelines per CTA (measured: one TMA ring + one MMA thread
-//                      per SM tops out near 4.9 TB/s, two reach the HBM limit): warps 0/1 stream
-//                      weights, warps 2/3 issue tcgen05.mma (accumulators in TMEM, double
-//                      buffered per pipeline), warps 4/5 TMA-load the activation operand, warps
-//                      6-9 drain TMEM to split-K partial sums (stream-K partition over 2 x grid
+//                      per SM tops out near 4.9 TB/s, two reach the HBM limit): warp 0
+//                      streams weights, warps 1/2 issue tcgen05.mma (accumulators in TMEM,
+//                      double buffered per pipeline), warp 3 TMA-loads the activation
+//                      operand, warps 4-7 drain TMEM to split-K partial sums (stream-K partition over 2 x grid
 //                      "virtual CTAs": every pipeline gets the same number of 128x64 weight
 //                      blocks, +-1), or, for the exit head, to top-2 records (there the two
 //                      pipelines take the two halves of each tile's K range);
-//   element-wise phase warps 2-9 of all CTAs: sum the partial slots in slot order, then
+//   element-wise phase warps 1-7 of all CTAs: sum the partial slots in slot order, then
 //                      RoPE + KV append / residual + gain + hi-lo split / SiLU*up / split merge;
-//   attention phase    warp 5 stages KV pages by TMA, warps 6-9 run the tiled attention;
+//   attention phase    warp 3 stages KV pages by TMA, warps 4-7 run the tiled attention;
 //   final phase        CTA b reduces sequence b's top-2 records and applies LeadingSubstringVerify.
 //
 // RMSNorm is applied as y = W (g .* x) / rms(x): the projection runs on g .* x and the row's
@@ -36,11 +36,17 @@
 
 namespace hispec {
 
-constexpr int kMegaThreads = 320;
+// Eight warps, two per scheduler partition: with ten, a partition with three warps limits every thread to
+// 168 registers, and the spills that caused cost every phase a memory round trip.
+constexpr int kMegaThreads = 256;
 constexpr int kMegaMaxStages = 8;  // per pipeline
 constexpr int kMegaMaxBatch = 64;
-constexpr int kMegaWorkers = 256;  // threads of warps 2..9
-constexpr int kMegaLeader = 64;    // warp 2 lane 0
+constexpr int kMegaWorkers = 224;  // threads of warps 1..7
+constexpr int kMegaLeader = 32;    // warp 1 lane 0
+// warp 0: one thread streams the weights of both pipelines; warps 1/2: tcgen05.mma of pipelines 0/1; warp 3:
+// activation operand of both pipelines and attention pages; warps 4..7: accumulator drain / attention tiles.
+// Warps 1..7 are the workers of the element-wise phases.
+constexpr int kWarpMma0 = 1, kWarpX = 3, kWarpEpi0 = 4;
 constexpr int kMegaAccCols = 128;  // TMEM columns per accumulator buffer (2 pipelines x 2 buffers)
 constexpr int kEwChunk = 256;      // columns per element-wise work item (one warp, 8 per lane)
 constexpr int kSsqChunk = 128;     // columns per sum-of-squares record
@@ -654,7 +660,7 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
         if (chunk < 1) chunk = 1;
         const int pg0 = split * chunk, pg1 = min(pg0 + chunk, total_pages);
         const int n_pg = (nr > 0 && pg1 > pg0) ? pg1 - pg0 : 0;
-        if (warp == 5) {
+        if (warp == kWarpX) {
             MEGA_STAMP(10);
             for (int i0 = 0; i0 < n_pg; i0 += 32) {
                 const int my = i0 + lane;
@@ -681,9 +687,9 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                 }
             }
             MEGA_STAMP(12);
-        } else if (warp >= 6) {
+        } else if (warp >= kWarpEpi0) {
             MEGA_STAMP(20);
-            const int cw = warp - 6;
+            const int cw = warp - kWarpEpi0;
             const int r_lo = mg * 64 + cw * 16 + (lane >> 2), r_hi = r_lo + 8;
             const int j_lo = r_lo / m.G, g_lo = r_lo % m.G, j_hi = r_hi / m.G, g_hi = r_hi % m.G;
             const bool v_lo = cw < m.mt && r_lo < QR && j_lo < nr, v_hi = cw < m.mt && r_hi < QR && j_hi < nr;
@@ -866,43 +872,108 @@ struct WCursor {
     }
 };
 
-// warps 0 and 1, one thread each: every weight block of the call that belongs to pipeline p, in
-// consumption order, into that pipeline's ring -- across projection and phase boundaries
-__device__ __forceinline__ void mega_w_producer(const MegaArgs &m, int p, const MegaRing &ring, MegaShared &sh) {
-    volatile int *ab = &sh.abort_flag;
-    WCursor ld(&m, &sh, p);
+// Both polling loops below serve the two pipelines from ONE thread with non-blocking tests: two lanes of a
+// warp that spin in separate loops are not scheduled fairly (one pipeline starves), and a third warp per
+// scheduler partition would cap every thread at 168 registers.
+__device__ __forceinline__ bool mega_poll_idle(uint32_t &idle, bool did, volatile int *ab, uint32_t *status) {
+    if (did) { idle = 0; return true; }
+    if (++idle >= (1u << 28)) { *ab = 1; atomicOr(status, HISPEC_ST_TIMEOUT); return false; }
+    if ((idle & 65535u) == 0u && *ab) return false;
+    return true;
+}
+
+// warp 0, one thread: every weight block of the call, per pipeline in consumption order, into that
+// pipeline's ring -- across projection and phase boundaries.  The first block of a projection is held back
+// until the previous projection's last block has LANDED: when the ring frees up at the end of a phase every
+// SM issues a ring's worth of loads at once, and without the gate the tail blocks the running phase still
+// waits for queue behind 24 MB of the next phase's data (measured: +1.5 to 3 us per phase).
+struct WLane {
+    WCursor ld;
     RingPos pos;
+    int cur_gi;
+    uint32_t last_bar, last_ph;
+    bool gate;
+    __device__ WLane(const MegaArgs *m, const MegaShared *sh, int p) : ld(m, sh, p), cur_gi(0), last_bar(0), last_ph(0), gate(false) {
+        cur_gi = ld.gi;
+    }
+};
+__device__ __forceinline__ bool mega_w_issue(const MegaArgs &m, int p, WLane &w, const MegaRing &ring, MegaShared &sh, uint64_t policy) {
+    if (!w.ld.valid) return false;
+    if (w.gate) {
+        if (!mbar_test_wait(w.last_bar, w.last_ph)) return false;
+        w.gate = false;
+    }
+    if (!mbar_test_wait(smem_u32(&sh.empty[p][w.pos.s]), w.pos.ph ^ 1u)) return false;
+#ifdef HISPEC_STAMPS
+    if (p == 0 && w.ld.kb == sh.segs[w.ld.kind()][0].kb0[0] && w.ld.si == 0) MEGA_STAMP(80 + w.ld.kind());
+#endif
+    const uint32_t fb = smem_u32(&sh.w_full[p][w.pos.s]);
+    mbar_expect_tx(fb, kWTileBytes);
+    tma_load_2d_stream(ring.base + w.pos.s * ring.stage_bytes, &w.ld.gemm()->tmW, w.ld.kb * kTileK, w.ld.tile * kWeightTileRows, fb,
+                       policy);
+    w.last_bar = fb;
+    w.last_ph = w.pos.ph;
+    w.ld.advance();
+    w.pos.advance(ring.stages);
+    if (w.ld.valid && w.ld.gi != w.cur_gi) { w.cur_gi = w.ld.gi; w.gate = true; }
+    return true;
+}
+__device__ __forceinline__ void mega_w_producer(const MegaArgs &m, const MegaRing *ring, MegaShared &sh) {
+    volatile int *ab = &sh.abort_flag;
+    WLane w0(&m, &sh, 0), w1(&m, &sh, 1);
     // weights are read exactly once per call: mark their lines evict-first so that they do not push the
     // partial sums, activations and KV pages (which are re-read) out of L2
     const uint64_t policy = l2_policy_evict_first();
-    while (ld.valid) {
-        if (!mbar_wait(smem_u32(&sh.empty[p][pos.s]), pos.ph ^ 1u, ab, m.status)) return;
-        const uint32_t fb = smem_u32(&sh.w_full[p][pos.s]);
-        mbar_expect_tx(fb, kWTileBytes);
-        const MegaGemm *g = ld.gemm();
-        tma_load_2d_stream(ring.base + pos.s * ring.stage_bytes, &g->tmW, ld.kb * kTileK, ld.tile * kWeightTileRows, fb, policy);
-        ld.advance();
-        pos.advance(ring.stages);
+    uint32_t idle = 0;
+    while (w0.ld.valid || w1.ld.valid) {
+        const bool d0 = mega_w_issue(m, 0, w0, ring[0], sh, policy);
+        const bool d1 = mega_w_issue(m, 1, w1, ring[1], sh, policy);
+        if (!mega_poll_idle(idle, d0 || d1, ab, m.status)) return;
     }
 }
 
-__device__ __forceinline__ bool mega_x_load(int kind, int p, const CUtensorMap *tmX, const MegaRing &ring,
-                                            MegaShared &sh, RingPos &pos, uint32_t *status) {
+// warp 3, one thread: the activation operand of both pipelines' k-blocks of one projection phase
+struct XCursor {
+    const SegList *L;
+    int i, kb;
+    bool valid;
+    __device__ XCursor(const SegList *L_) : L(L_), i(0), kb(0), valid(L_->n > 0) {
+        if (valid) kb = L->kb0[0];
+        skip();
+    }
+    __device__ void skip() {
+        while (valid && kb >= L->kb1[i]) {
+            if (++i >= L->n) valid = false; else kb = L->kb0[i];
+        }
+    }
+    __device__ void advance() { ++kb; skip(); }
+};
+__device__ __forceinline__ bool mega_x_load(int kind, const CUtensorMap *tmX, const MegaRing *ring, MegaShared &sh,
+                                            RingPos *pos, uint32_t *status) {
     volatile int *ab = &sh.abort_flag;
-    const SegList &L = sh.segs[kind][p];
+    XCursor c0(&sh.segs[kind][0]), c1(&sh.segs[kind][1]);
     uint64_t policy;   // the activation operand is re-read by every CTA: keep it in L2
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
-    for (int i = 0; i < L.n; ++i) {
-        for (int kb = L.kb0[i]; kb < L.kb1[i]; ++kb) {
-            if (!mbar_wait(smem_u32(&sh.empty[p][pos.s]), pos.ph ^ 1u, ab, status)) return false;
-            const uint32_t fb = smem_u32(&sh.x_full[p][pos.s]);
-            mbar_expect_tx(fb, ring.x_bytes);
-            asm volatile(
-                "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
-                ::"r"(ring.base + pos.s * ring.stage_bytes + kWTileBytes), "l"(tmX), "r"(kb * kTileK), "r"(0), "r"(0), "r"(fb),
-                "l"(policy) : "memory");
-            pos.advance(ring.stages);
+    uint32_t idle = 0;
+    while (c0.valid || c1.valid) {
+        bool did = false;
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            XCursor &c = p ? c1 : c0;
+            RingPos &ps = pos[p];
+            if (c.valid && mbar_test_wait(smem_u32(&sh.empty[p][ps.s]), ps.ph ^ 1u)) {
+                const uint32_t fb = smem_u32(&sh.x_full[p][ps.s]);
+                mbar_expect_tx(fb, ring[p].x_bytes);
+                asm volatile(
+                    "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+                    ::"r"(ring[p].base + ps.s * ring[p].stage_bytes + kWTileBytes), "l"(tmX), "r"(c.kb * kTileK), "r"(0), "r"(0),
+                    "r"(fb), "l"(policy) : "memory");
+                c.advance();
+                ps.advance(ring[p].stages);
+                did = true;
+            }
         }
+        if (!mega_poll_idle(idle, did, ab, status)) return false;
     }
     return true;
 }
@@ -949,7 +1020,7 @@ __device__ __forceinline__ void mega_acc_ld8(uint32_t taddr, int c0, int t_box, 
     }
 }
 
-// warps 6..9, split-K projections: drain the accumulators of both pipelines' segments, alternating
+// warps 4..7, split-K projections: drain the accumulators of both pipelines' segments, alternating
 __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, const MegaArgs &m, MegaShared &sh,
                                                    uint32_t *seg_it, int warp, int lane) {
     volatile int *ab = &sh.abort_flag;
@@ -994,7 +1065,7 @@ __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, 
     return true;
 }
 
-// warps 6..9, exit head: each tile's accumulator is the sum of the two pipelines' K halves; every
+// warps 4..7, exit head: each tile's accumulator is the sum of the two pipelines' K halves; every
 // column (activation row) is reduced to its top-2 over this warp's 32 vocabulary entries
 __device__ __forceinline__ bool mega_epilogue_head(const MegaGemm *g, const MegaArgs &m, MegaShared &sh,
                                                    uint32_t *seg_it, int warp, int lane) {
@@ -1051,7 +1122,7 @@ __device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b) {
     const StageArgs &a = m.a;
     const AcceptArgs &r = m.r;
     const int nr = sh.nr[b];
-    const int wt = threadIdx.x - kMegaLeader, lane = threadIdx.x & 31, w = (threadIdx.x >> 5) - 2;
+    const int wt = threadIdx.x - kMegaLeader, lane = threadIdx.x & 31, w = (threadIdx.x >> 5) - 1;
     const int n_rec = m.head->tiles * 4;
     for (int j = 0; j < nr; ++j) {
         const int t = b * a.R_pad + j;
@@ -1174,24 +1245,24 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
-    if (warp < 2) {
-        // ---- weight producers: the whole call's weight blocks of pipeline `warp`, in consumption order
-        if (lane == 0) mega_w_producer(m, warp, ring[warp], sh);
+    if (warp == 0) {
+        // ---- weight producer: the whole call's weight blocks of both pipelines, in consumption order
+        if (lane == 0) mega_w_producer(m, ring, sh);
     } else {
-        const int gw = (warp - 2) * gridDim.x + blockIdx.x, ngw = (kMegaWorkers / 32) * gridDim.x;
+        const int gw = (warp - 1) * gridDim.x + blockIdx.x, ngw = (kMegaWorkers / 32) * gridDim.x;
         uint32_t seg_it[2] = {0, 0}, pg_it = 0;   // per-thread progress counters of the role loops
-        RingPos pos;
+        RingPos pos, xpos[2];
         const CUtensorMap *tmX[3] = {&tmXd, &tmXo, &tmXf};
         // `head` is a compile-time tag: the layer loop holds ONE copy of the projection roles for its four
         // projections (a copy per projection made a layer's code larger than the instruction cache)
         auto gemm_phase = [&](const MegaGemm *g, int kind, int xbuf, auto head) {
             MEGA_STAMP(40 + kind);
-            if (warp == 2 || warp == 3) {
-                const int p = warp - 2;
+            if (warp == kWarpMma0 || warp == kWarpMma0 + 1) {
+                const int p = warp - kWarpMma0;
                 if (lane == 0) mega_mma(m, kind, p, ncols, ring[p], sh, pos, seg_it[p], m.status);
-            } else if (warp == 4 || warp == 5) {
-                const int p = warp - 4;
-                if (lane == 0) mega_x_load(kind, p, tmX[xbuf], ring[p], sh, pos, m.status);
+            } else if (warp == kWarpX) {
+                if (lane == 0) mega_x_load(kind, tmX[xbuf], ring, sh, xpos, m.status);
+                __syncwarp();
             } else {
                 if constexpr (decltype(head)::value) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
                 else mega_epilogue_part(g, kind, m, sh, seg_it, warp, lane);
