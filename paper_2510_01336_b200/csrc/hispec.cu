@@ -299,6 +299,8 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
                 if (v > worst) worst = v;
             }
         c->attn_max_splits = (int)(worst / ((size_t)d.max_batch * d.max_rows_per_seq)) + 1;
+        // the persistent kernel keeps up to 32 records per (row, head): key splits x warp groups
+        if (worst < (size_t)32 * d.max_batch * d.max_rows_per_seq) worst = (size_t)32 * d.max_batch * d.max_rows_per_seq;
         c->attn_part_floats = worst * d.n_q_heads * (d.head_dim + 4);   // records padded to 16 bytes by the persistent kernel
     }
     auto alloc = [&](void **p, size_t bytes) { return cudaMalloc(p, bytes ? bytes : 16) == cudaSuccess; };
@@ -650,8 +652,10 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         if (m.n_splits < by_len) m.n_splits = by_len;
     }
     if (m.n_splits < 1) m.n_splits = 1;
-    if (m.n_splits > 16) m.n_splits = 16;   // one load batch in the split merge
-    if ((size_t)m.n_splits * T_pad * d.n_q_heads * (d.head_dim + kAttnRecPad) > c->attn_part_floats) return 1;
+    if (m.n_splits > 16) m.n_splits = 16;
+    m.ngrp = m.mt == 1 ? 4 : (m.mt == 2 ? 2 : 1);
+    if (m.n_splits * m.ngrp > 32) m.ngrp = 32 / m.n_splits;   // one load batch in the split merge (16 splits: ngrp <= 2)
+    if ((size_t)m.n_splits * m.ngrp * T_pad * d.n_q_heads * (d.head_dim + kAttnRecPad) > c->attn_part_floats) return 1;
     m.scale_log2 = (1.0f / sqrtf((float)d.head_dim)) * 1.4426950408889634f;
     m.r.len_d = kv.len_draft; m.r.len_i = kv.len_inter; m.r.len_f = kv.len_target;
     m.r.draft_tokens = sc.draft_tokens; m.r.token_stride = sc.token_stride; m.r.out_stride = sc.out_stride;

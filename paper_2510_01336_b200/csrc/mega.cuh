@@ -82,6 +82,7 @@ struct MegaArgs {
     const double *inv_freq;
     float2 *rope;            // [T_pad][hd / 2] (cos, sin) of each row's position, filled in the first phase
     int n_splits, n_mg, mt, G;
+    int ngrp;                // warp groups that share an attention item's pages (4, 2 or 1); records per (row, head) = n_splits * ngrp
     float scale_log2;
     AcceptArgs r;
     int32_t *argmax_ws;
@@ -466,13 +467,20 @@ __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, c
     }
 }
 
-// 1 / rms of row t, lanes fetching the chunk sums in parallel; same value in every lane
-__device__ __forceinline__ float mega_inv_rms_warp(const MegaArgs &m, int t, int lane) {
+// 1 / rms of row t in two steps, so that the caller can put its other loads between them and pay one
+// memory round trip instead of two: lanes fetch the chunk sums (no use of the values yet) ...
+__device__ __forceinline__ float mega_ssq_fetch(const MegaArgs &m, int t, int lane) {
     const int nch = (m.d + kSsqChunk - 1) / kSsqChunk;
     float s = 0.f;
     for (int c = lane; c < nch; c += 32) s += m.ssq[(size_t)t * nch + c];
-    s = warp_sum(s);
-    return rsqrtf(s / (float)m.d + m.eps);
+    return s;
+}
+// ... and reduce them; same value in every lane
+__device__ __forceinline__ float mega_inv_rms_finish(const MegaArgs &m, float s) {
+    return rsqrtf(warp_sum(s) / (float)m.d + m.eps);
+}
+__device__ __forceinline__ float mega_inv_rms_warp(const MegaArgs &m, int t, int lane) {
+    return mega_inv_rms_finish(m, mega_ssq_fetch(m, t, lane));
 }
 
 // a3: q,k,v = projection / rms; rotate q,k; append K,V to the sequence's pages.  One warp per (row, head).
@@ -487,7 +495,7 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
                 for (int i = lane; i < hd; i += 32) m.q[(size_t)t * nq + h * hd + i] = 0.f;
             continue;
         }
-        const float inv = mega_inv_rms_warp(m, t, lane);
+        const float ssq = mega_ssq_fetch(m, t, lane);
         const int pos = sh.p0[b] + j;
         const int lp = pos / a.page_size, slot = pos % a.page_size;
         const long long page = m.block_table[(size_t)b * a.max_pages + lp];
@@ -498,26 +506,41 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         int first, ns;
         mega_slots((h * hd) / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
         const float *pr = m.part + (size_t)t * g.N + h * hd;
-        if (h < m.hq + m.hkv) {
-            for (int i = lane; i < half; i += 32) {
-                const float2 cs = m.rope[(size_t)t * half + i];
-                float x0 = 0.f, x1 = 0.f;
-                // slots eight at a time: all sixteen loads of a batch are in flight together; slots past the
-                // last one re-read it with weight zero, so the order of the sum is the slot order
-                for (int s0 = 0; s0 < ns; s0 += 8) {
-                    float u0[8], u1[8];
+        // lane l owns columns l + 32 e of the head (e < hd / 32; hd is 64 or 128).  Every load of the item --
+        // chunk sums, rotary pair, up to eight slots of each column -- is issued before the first use.
+        const int ne = hd >> 5;
+        const bool rot = h < m.hq + m.hkv;
+        float2 cs[2] = {make_float2(1.f, 0.f), make_float2(1.f, 0.f)};
+        if (rot) {
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int sidx = s0 + u < ns ? s0 + u : ns - 1;
-                        u0[u] = pr[sidx * stride + i];
-                        u1[u] = pr[sidx * stride + i + half];
-                    }
+            for (int e = 0; e < 2; ++e)
+                if (e < ne / 2) cs[e] = m.rope[(size_t)t * half + lane + 32 * e];
+        }
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int s0 = 0; s0 < ns; s0 += 8) {
+            float u[4][8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        if (s0 + u < ns) { x0 += u0[u]; x1 += u1[u]; }
+            for (int e = 0; e < 4; ++e)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int sidx = s0 + k < ns ? s0 + k : ns - 1;   // past the last slot: re-read it, weight zero
+                    u[e][k] = e < ne ? pr[sidx * stride + lane + 32 * e] : 0.f;
                 }
-                x0 *= inv; x1 *= inv;
-                const float c = cs.x, sf = cs.y;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (s0 + k < ns) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) x[e] += u[e][k];   // slot order
+                }
+        }
+        const float inv = mega_inv_rms_finish(m, ssq);
+        if (rot) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                if (e >= ne / 2) break;
+                const int i = lane + 32 * e;
+                const float x0 = x[e] * inv, x1 = (ne == 4 ? x[e + 2] : x[e + 1]) * inv;
+                const float c = cs[e].x, sf = cs[e].y;
                 const float r0 = x0 * c - x1 * sf, r1 = x1 * c + x0 * sf;
                 if (h < m.hq) {
                     m.q[(size_t)t * nq + h * hd + i] = r0;
@@ -531,24 +554,9 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         } else if (page_ok) {
             const int vh = h - m.hq - m.hkv;
             const size_t o = page_base + ((size_t)vh * a.page_size + slot) * hd;
-            for (int i = lane; i < hd; i += 64) {
-                float v0 = 0.f, v1 = 0.f;
-                const int i1 = i + 32 < hd ? i + 32 : i;
-                for (int s0 = 0; s0 < ns; s0 += 8) {
-                    float u0[8], u1[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int sidx = s0 + u < ns ? s0 + u : ns - 1;
-                        u0[u] = pr[sidx * stride + i];
-                        u1[u] = pr[sidx * stride + i1];
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        if (s0 + u < ns) { v0 += u0[u]; v1 += u1[u]; }
-                }
-                m.v_pages[o + i] = __float2bfloat16_rn(inv * v0);
-                if (i + 32 < hd) m.v_pages[o + i + 32] = __float2bfloat16_rn(inv * v1);
-            }
+            for (int e = 0; e < 4; ++e)
+                if (e < ne) m.v_pages[o + lane + 32 * e] = __float2bfloat16_rn(inv * x[e]);
         }
     }
 }
@@ -559,11 +567,14 @@ __device__ void ew_silu(const MegaArgs &m, const MegaGemm &g, int gw, int ngw, i
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
         const int t = item / nch, ch = item % nch;
         const int c = ch * kEwChunk + lane * 8;
-        const float inv = mega_inv_rms_warp(m, t, lane);
-        if (c >= m.ffn) continue;
+        const float ssq = mega_ssq_fetch(m, t, lane);
         float gt[8], up[8], v[8];
-        sum_slots8(m, g, t, c, gt);
-        sum_slots8(m, g, t, m.ffn + c, up);
+        if (c < m.ffn) {
+            sum_slots8(m, g, t, c, gt);
+            sum_slots8(m, g, t, m.ffn + c, up);
+        }
+        const float inv = mega_inv_rms_finish(m, ssq);
+        if (c >= m.ffn) continue;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const float gg = gt[i] * inv;
@@ -591,10 +602,11 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
         float inv = 0.f;
         if (j < sh.nr[b]) {
-            const float *base = m.attn_part + ((size_t)t * m.hq + h) * m.n_splits * REC;
+            const int n_rec = m.n_splits * m.ngrp;
+            const float *base = m.attn_part + ((size_t)t * m.hq + h) * n_rec * REC;
             float L = 0.f, M = -INFINITY;
-            for (int s0 = 0; s0 < m.n_splits; s0 += 32) {
-                const int cnt = min(32, m.n_splits - s0);
+            for (int s0 = 0; s0 < n_rec; s0 += 32) {
+                const int cnt = min(32, n_rec - s0);
                 float ms = -INFINITY, ls = 0.f;   // lane u holds (max, sum) of split s0 + u
                 if (lane < cnt) {
                     const float2 ml = *reinterpret_cast<const float2 *>(base + (size_t)(s0 + lane) * REC + HD);
@@ -689,7 +701,10 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             MEGA_STAMP(12);
         } else if (warp >= kWarpEpi0) {
             MEGA_STAMP(20);
-            const int cw = warp - kWarpEpi0;
+            // With one or two 16-row tiles in the item the four warps form 4 or 2 groups that take the item's
+            // pages in turn; each group leaves its own record, combined with the key splits by the merge.
+            const int mtp = 4 / m.ngrp;
+            const int cw = (warp - kWarpEpi0) % mtp, grp = (warp - kWarpEpi0) / mtp;
             const int r_lo = mg * 64 + cw * 16 + (lane >> 2), r_hi = r_lo + 8;
             const int j_lo = r_lo / m.G, g_lo = r_lo % m.G, j_hi = r_hi / m.G, g_hi = r_hi % m.G;
             const bool v_lo = cw < m.mt && r_lo < QR && j_lo < nr, v_hi = cw < m.mt && r_hi < QR && j_hi < nr;
@@ -728,11 +743,15 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                 ok = a_wait(a_smem_u32(&sh.a_full[s]), ph, abort_flag, m.status);
                 if (!ok) break;
                 MEGA_STAMP(22);
-                if (active) {
+                if (active && (i % m.ngrp) == grp) {
                     const uint32_t sk = sm_attn + s * 2 * TILE, sv = sk + TILE;
-                    float sc[2][4];
+                    // four independent accumulator chains (2 key tiles x hi/lo query planes), added at the end
+                    float sc[2][4], sl[2][4];
 #pragma unroll
-                    for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+                    for (int n = 0; n < 2; ++n) {
+                        sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+                        sl[n][0] = sl[n][1] = sl[n][2] = sl[n][3] = 0.f;
+                    }
                     const int mat = lane >> 3, rin = lane & 7;
 #pragma unroll
                     for (int ks = 0; ks < KS; ++ks) {
@@ -742,10 +761,14 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                         uint32_t kb[4];
                         ldmatrix_x4(addr, kb);
                         mma_bf16_16816(sc[0], qh[ks], kb[0], kb[1]);
-                        mma_bf16_16816(sc[0], ql[ks], kb[0], kb[1]);
+                        mma_bf16_16816(sl[0], ql[ks], kb[0], kb[1]);
                         mma_bf16_16816(sc[1], qh[ks], kb[2], kb[3]);
-                        mma_bf16_16816(sc[1], ql[ks], kb[2], kb[3]);
+                        mma_bf16_16816(sl[1], ql[ks], kb[2], kb[3]);
                     }
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) sc[n][e] += sl[n][e];
                     const int key0 = (pg0 + i) * 16;
                     float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
@@ -797,13 +820,13 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
             if (!ok) { l_lo = l_hi = 0.f; m_lo = m_hi = -INFINITY; }
             if (v_lo) {
-                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_lo) * m.hq + kvh * m.G + g_lo) * m.n_splits + split) * (HD + kAttnRecPad));
+                float *dst = m.attn_part + (((((size_t)(b * a.R_pad + j_lo) * m.hq + kvh * m.G + g_lo) * m.n_splits + split) * m.ngrp + grp) * (HD + kAttnRecPad));
 #pragma unroll
                 for (int n = 0; n < NT; ++n) *reinterpret_cast<float2 *>(dst + n * 8 + c2) = make_float2(o[n][0], o[n][1]);
                 if ((lane & 3) == 0) { dst[HD] = m_lo; dst[HD + 1] = l_lo; }
             }
             if (v_hi) {
-                float *dst = m.attn_part + ((((size_t)(b * a.R_pad + j_hi) * m.hq + kvh * m.G + g_hi) * m.n_splits + split) * (HD + kAttnRecPad));
+                float *dst = m.attn_part + (((((size_t)(b * a.R_pad + j_hi) * m.hq + kvh * m.G + g_hi) * m.n_splits + split) * m.ngrp + grp) * (HD + kAttnRecPad));
 #pragma unroll
                 for (int n = 0; n < NT; ++n) *reinterpret_cast<float2 *>(dst + n * 8 + c2) = make_float2(o[n][2], o[n][3]);
                 if ((lane & 3) == 0) { dst[HD] = m_hi; dst[HD + 1] = l_hi; }
