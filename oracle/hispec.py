@@ -266,6 +266,31 @@ class GenStats:
     committed: int = 0
 
 
+@dataclass
+class AdaptiveSpec:
+    """Bounds and thresholds of one adaptive hyper-parameter (App. J)."""
+    tau_high: float
+    tau_low: float
+    n_min: int
+    n_max: int
+
+
+# App. J: N_d follows the acceptance rate of the intermediate verifier (thresholds 0.8 / 0.5, bounds [1, 3]),
+# N_i that of the final layer (thresholds 0.8 / 0.3, bounds [3, 8]).
+ADAPT_ND_PAPER = AdaptiveSpec(0.8, 0.5, 1, 3)
+ADAPT_NI_PAPER = AdaptiveSpec(0.8, 0.3, 3, 8)
+
+
+def adaptive_step(n: int, alpha: float, spec: AdaptiveSpec) -> int:
+    """Next value of N_d (or N_i) given this step's acceptance rate alpha (App. J, the two update equations):
+    one more if alpha >= tau_high (capped at n_max), one less if alpha < tau_low (floored at n_min), else unchanged."""
+    if alpha >= spec.tau_high:
+        return min(spec.n_max, n + 1)
+    if alpha < spec.tau_low:
+        return max(spec.n_min, n - 1)
+    return n
+
+
 class HiSpecOracle:
     def __init__(self, model: OracleModel, L_d: int, L_i: int, L_f: int):
         assert 0 < L_d < L_i < L_f <= model.n_layers
@@ -419,7 +444,9 @@ class HiSpecOracle:
     def hispec_generate(self, prompt: Sequence[int], n_gen: int, N_d: int, *, N_i: Optional[int] = None,
                         rounds: Optional[int] = None, bonus_inter: bool = True, bonus_target: bool = False,
                         draft_override: Optional[Callable[[int, int], int]] = None, observer=None,
-                        stats: Optional[GenStats] = None, rows_cap: Optional[int] = None) -> List[int]:
+                        stats: Optional[GenStats] = None, rows_cap: Optional[int] = None,
+                        adapt_nd: Optional[AdaptiveSpec] = None, adapt_ni: Optional[AdaptiveSpec] = None,
+                        schedule: Optional[list] = None) -> List[int]:
         """Algorithm 2.  The inner loop drafts and verifies at L_i until the
         trigger fires -- |V| >= N_i (the paper's dynamic policy, Sec. 3.4) or a
         fixed number of `rounds` -- then L_f verifies V.  Returns the n_gen
@@ -431,11 +458,17 @@ class HiSpecOracle:
         (adversarial or acceptance-shaped drafts); the output must not depend on it.
         `observer.before(kind, st, seq_tokens, **kw)` / `.after(kind, st, out)`
         see every stage call (kind in {"draft", "verify_i", "verify_t"}).
+        `adapt_nd` / `adapt_ni` (App. J) re-choose N_d after every intermediate verification from its
+        acceptance rate (accepted / drafted) and N_i after every target verification from its acceptance rate
+        (accepted / |V|); `schedule` collects ("i", N_d, accepted) and ("t", N_i, |V|, accepted) records.
         """
         assert (N_i is None) != (rounds is None)
+        assert adapt_ni is None or N_i is not None
         stats = stats if stats is not None else GenStats()
-        per_round = N_d + 1
-        cap_rows = rows_cap or ((rounds * per_round if rounds else N_i + per_round) + 2)
+        nd_max = adapt_nd.n_max if adapt_nd else N_d
+        ni_max = adapt_ni.n_max if adapt_ni else N_i
+        per_round = max(N_d, nd_max) + 1
+        cap_rows = rows_cap or ((rounds * per_round if rounds else max(N_i, ni_max) + per_round) + 2)
         st = self.new_state(len(prompt) + n_gen + cap_rows + 2, cap_rows)
         pending = self.prefill(st, prompt).argmax_ids[0]
         x = list(int(t) for t in prompt) + [pending]
@@ -460,6 +493,10 @@ class HiSpecOracle:
                 V += Vhat
                 pending = V[-1]
                 r += 1
+                if schedule is not None:
+                    schedule.append(("i", N_d, int(out.n_accepted)))
+                if adapt_nd is not None:
+                    N_d = adaptive_step(N_d, out.n_accepted / len(S), adapt_nd)
             R = len(V)
             if bonus_target:  # catch V's last token up through [0, L_i) so that L_f can emit a bonus token
                 obs_b("draft", st, x + V, token=pending)
@@ -479,6 +516,10 @@ class HiSpecOracle:
             F, _ = leading_substring_verify(V, out.argmax_ids)
             x += F
             pending = F[-1]
+            if schedule is not None:
+                schedule.append(("t", N_i, len(V), int(out.n_accepted)))
+            if adapt_ni is not None:
+                N_i = adaptive_step(N_i, out.n_accepted / len(V), adapt_ni)
         stats.committed = min(len(x) - n0, n_gen)
         return x[n0: n0 + n_gen]
 

@@ -176,6 +176,97 @@ class HiSpecDynamicLoop(HiSpecLoop):
             self.rounds = rounds
 
 
+@dataclass
+class AdaptiveRule:
+    """One adaptive hyper-parameter (App. J): the value moves up by one when the step's acceptance rate
+    reaches tau_high, down by one when it falls below tau_low, and stays inside [n_min, n_max]."""
+    tau_high: float
+    tau_low: float
+    n_min: int
+    n_max: int
+
+    def next(self, n: int, alpha: float) -> int:
+        if alpha >= self.tau_high:
+            return min(self.n_max, n + 1)
+        if alpha < self.tau_low:
+            return max(self.n_min, n - 1)
+        return n
+
+
+ND_RULE_PAPER = AdaptiveRule(0.8, 0.5, 1, 3)   # N_d from the intermediate verifier's acceptance rate
+NI_RULE_PAPER = AdaptiveRule(0.8, 0.3, 3, 8)   # N_i from the final layer's acceptance rate
+
+
+class HiSpecAdaptiveLoop(HiSpecDynamicLoop):
+    """Algorithm 2 with the adaptive choice of N_d and N_i (App. J).  N_d is re-chosen after every
+    intermediate verification, N_i after every target verification; with several sequences in the batch the
+    acceptance rate of a step is the mean over the sequences.  The draft block keeps its widest layout
+    (stride nd_rule.n_max), so a change of N_d moves no buffer."""
+
+    def __init__(self, ctx, st, batch, N_d, N_i, nd_rule: Optional[AdaptiveRule] = ND_RULE_PAPER,
+                 ni_rule: Optional[AdaptiveRule] = NI_RULE_PAPER, device="cuda"):
+        nd_max = max(N_d, nd_rule.n_max if nd_rule else N_d)
+        ni_max = max(N_i, ni_rule.n_max if ni_rule else N_i)
+        super().__init__(ctx, st, batch, nd_max, ni_max, device=device)
+        self.nd_rule, self.ni_rule = nd_rule, ni_rule
+        self.N_d_cur, self.N_i_cur = N_d, N_i
+        # every round commits at least one token to V, so N_i rounds always reach the trigger
+        i32 = lambda *sh: torch.zeros(sh, dtype=torch.int32, device=device)
+        while len(self.res_i) < ni_max:
+            r = binding.Result(i32(batch), i32(batch))
+            r.tentative, r.pending = self.V, self.pending
+            self.res_i.append(r)
+        self.rounds = len(self.res_i)
+        self.h_acc_i = torch.zeros((self.rounds, batch), dtype=torch.int32).pin_memory()
+        self.h_acc_round = torch.zeros(batch, dtype=torch.int32).pin_memory()
+        self.schedule: List[tuple] = []            # ("i", N_d, accepted...) / ("t", N_i, |V|..., accepted...) per step
+
+    def enqueue_super_round(self, stream=None):
+        ctx, st, B, W = self.ctx, self.st, self.B, self.N_d      # W: stride of the draft block
+        S_ptr = self.S.data_ptr()
+        s = stream if stream is not None else torch.cuda.current_stream()
+        self.rounds_used = 0
+        self._inter_acc = 0
+        for r in range(self.rounds):
+            n_d = self.N_d_cur
+            for j in range(n_d):
+                if j == 0:
+                    ctx.draft(st, self.pending, S_ptr, batch=B, in_stride=1, out_stride=W, stream=stream)
+                else:
+                    ctx.draft(st, S_ptr + 4 * (j - 1), S_ptr + 4 * j, batch=B, in_stride=W, out_stride=W, stream=stream)
+            ctx.draft(st, S_ptr + 4 * (n_d - 1), None, batch=B, in_stride=W, stream=stream)
+            ctx.verify_intermediate(st, self.S, None, None, self.res_i[r], stream=stream, k=n_d)
+            self.stats.draft_steps += n_d + 1
+            self.stats.inter_calls += 1
+            self.rounds_used += 1
+            with torch.cuda.stream(s):
+                self.h_len[0].copy_(st.len_inter, non_blocking=True)
+                self.h_len[1].copy_(st.len_target, non_blocking=True)
+                self.h_acc_round.copy_(self.res_i[r].n_accepted, non_blocking=True)
+            s.synchronize()
+            acc = self.h_acc_round.tolist()
+            self.schedule.append(("i", n_d, *acc))
+            if self.nd_rule is not None:
+                self.N_d_cur = self.nd_rule.next(n_d, sum(acc) / (B * n_d))
+            n_v = self.h_len[0] - self.h_len[1]
+            if int(n_v.min()) >= self.N_i_cur:   # every sequence has |V| >= N_i
+                break
+            if int(n_v.max()) + self.N_d_cur + 1 > ctx.max_rows - 1:   # no room for another round's rows
+                break
+        self._n_v = (self.h_len[0] - self.h_len[1]).tolist()
+        ctx.verify_target(st, self.V, None, None, self.res_t, stream=stream, k=ctx.max_rows - 1)
+        self.stats.target_calls += 1
+        self.stats.super_rounds += 1
+
+    def collect(self, stream=None):
+        new = super().collect(stream)
+        acc = self.h_acc.tolist()
+        self.schedule.append(("t", self.N_i_cur, *self._n_v, *acc))
+        if self.ni_rule is not None:
+            self.N_i_cur = self.ni_rule.next(self.N_i_cur, sum(acc) / max(1, sum(self._n_v)))
+        return new
+
+
 class SelfSpecLoop:
     """Algorithm 1 (single-stage self-speculation): N_d (+1) draft steps at L_d, then one verification of the
     block by the final layer -- hispec_verify_intermediate over [L_d, L_f) with the L_f exit."""

@@ -205,6 +205,46 @@ def test_tiny_dynamic_trigger_and_single_stage_loops_are_lossless():
     assert outs["dynamic"] == outs["ar"] and outs["selfspec"] == outs["ar"]
 
 
+def test_tiny_adaptive_parameters_loop_is_lossless():
+    """Adaptive N_d / N_i (App. J) free-running on the GPU: the output equals the GPU's own auto-regressive
+    greedy output, both parameters move, and the recorded schedule obeys the oracle's update rule."""
+    b = _binding()
+    from oracle import hispec as oh
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecAdaptiveLoop
+    shape = wl.TINY
+    scale = {l: 0.05 for l in range(shape.L_d, shape.L_f)}
+    wg = wl.make_weights(shape, resid_scale=scale).to("cuda")
+    n_prompt, n_gen = 64, 64
+    max_rows, max_pages = 14, (n_prompt + n_gen + 40) // 16 + 1
+    prompt = wl.make_tokens(shape, n_prompt).tolist()
+    bt = wl.make_block_table(shape, 1, max_pages)
+    ctx = b.Context(shape, wg, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    st = ctx.new_state(1, max_pages, bt)
+    loop = HiSpecAdaptiveLoop(ctx, st, 1, 2, 4)
+    loop.prefill([prompt])
+    toks = loop.generate(n_gen)[0]
+    assert ctx.status() == 0
+    ctx.close()
+    ctx2 = b.Context(shape, wg, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    st2 = ctx2.new_state(1, max_pages, bt)
+    ar = ARLoop(ctx2, st2, 1)
+    ar.prefill([prompt])
+    assert toks == ar.generate(n_gen)[0]
+    ctx2.close()
+    n_d, n_i = 2, 4
+    seen_d, seen_i = set(), set()
+    for rec in loop.schedule:
+        if rec[0] == "i":
+            assert rec[1] == n_d and 0 <= rec[2] <= n_d
+            seen_d.add(n_d)
+            n_d = oh.adaptive_step(n_d, rec[2] / rec[1], oh.ADAPT_ND_PAPER)
+        else:
+            assert rec[1] == n_i and rec[2] >= 1 and rec[3] <= rec[2]
+            seen_i.add(n_i)
+            n_i = oh.adaptive_step(n_i, rec[3] / rec[2], oh.ADAPT_NI_PAPER)
+    assert len(seen_d) > 1 and len(seen_i) > 1
+
+
 @pytest.mark.parametrize("flagname,B", [("tcgen05", 3), ("simt", 3), ("rowwarp-attn", 3), ("multi-kernel", 3),
                                         ("tcgen05", 20)])
 def test_batched_ragged_gqa_pages_permuted(flagname, B):
