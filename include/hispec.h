@@ -126,6 +126,10 @@ typedef struct {
     int32_t *pending;    /* optional device [batch]: the token that is pending after a verify call, i.e. the
                             last element of its result list: v_{a_b+1} if that row was computed, else the last
                             accepted block token; untouched for a sequence with no rows */
+    int32_t defer_accept; /* verify calls only.  Non-zero: compute the rows (KV appended, exit rows buffered,
+                            argmax_ids / top2 / logits written) but decide nothing -- n_accepted, next_token,
+                            tentative, pending and the three length counters stay as they were, for
+                            hispec_accept_rejection to decide on the same stream */
 } hispec_result;
 
 /* Create a context: validates the shape, copies the pointer tables, builds TMA descriptors for
@@ -194,6 +198,40 @@ int hispec_verify_target(hispec_ctx *ctx, void *stream, int layer_begin, int lay
  */
 int hispec_prefill(hispec_ctx *ctx, void *stream, const hispec_exits *exits, const hispec_kv *kv, int batch,
                    const int32_t *tokens, const int32_t *n_tokens, int max_tokens, int32_t *first_token);
+
+/*
+ * Rejection-sampling acceptance (App. G) for a verify call that ran with res->defer_accept: per sequence,
+ * for j = 0..n_draft-1 in order the block token S_{j+1} = draft_tokens[b * token_stride + j] is kept while
+ * u_accept[b * max_rows_per_seq + j] < min(1, q_j(S_{j+1}) / p_j(S_{j+1})); at the first failure the rest of
+ * the block is dropped and the next token is drawn from max(0, q_j - p_j) normalised; if every token is kept
+ * and the verifier computed one more row, the next token is drawn from that row's q.  Draws use inversion in
+ * vocabulary order with u_sample[b].  p_j = softmax(p_logits[b][j] / temperature) (the exit that proposed the
+ * block: rows written by the draft steps for stage 1, the rows kept by stage 1 for stage 2), q_j likewise
+ * from q_logits (the deferred call's res->logits); both device fp32 [batch][max_rows_per_seq][vocab].
+ * stage 1 = intermediate verification over [L_d, L_i), stage 2 = target verification over [L_i, L_f);
+ * n_rows / n_draft are taken from the length counters exactly as the verify calls do with NULL n_rows
+ * (k = the verify call's k).  Then the state transition of the verify call is applied with the sampled
+ * outcome: n_accepted, next_token, tentative, pending and the length counters as documented for
+ * hispec_verify_intermediate / hispec_verify_target.  Stage 1 also appends the q rows of the kept tokens and
+ * of the next token (rows 0..min(a, n_rows - 1)) to stage_logits [batch][max_rows_per_seq][vocab] at row
+ * len_inter - len_target (entry values): the proposal rows stage 2 needs.  stage_logits may be NULL.
+ * Probabilities are formed in fp32.  The paper has the rule (App. G); the entry point, its arguments and the
+ * uniforms-as-inputs convention are this library's.  Returns HISPEC_EINVAL on bad arguments; state errors go
+ * to the status word.
+ */
+int hispec_accept_rejection(hispec_ctx *ctx, void *stream, int stage, const hispec_exits *exits,
+                            const hispec_kv *kv, int batch, const int32_t *draft_tokens, int token_stride, int k,
+                            const float *p_logits, const float *q_logits, const float *u_accept,
+                            const float *u_sample, float temperature, float *stage_logits,
+                            const hispec_result *res);
+
+/*
+ * Draw one token per sequence from softmax(logits[b * row_stride ...] / temperature) by inversion in
+ * vocabulary order with u[b] (device fp32 [batch], in [0,1)); the token goes to out_tokens[b * out_stride].
+ * Used to sample draft tokens from the logits a draft step wrote (App. G: drafts are sampled from p_{L_d}).
+ */
+int hispec_sample(hispec_ctx *ctx, void *stream, int batch, const float *logits, int64_t row_stride,
+                  const float *u, float temperature, int32_t *out_tokens, int out_stride);
 
 /* Synchronises `stream`, copies the device status word to *host_out and clears it. */
 int hispec_device_status(hispec_ctx *ctx, void *stream, uint32_t *host_out);

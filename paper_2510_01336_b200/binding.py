@@ -28,7 +28,7 @@ ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 EXPORTS = ["hispec_create", "hispec_destroy", "hispec_draft", "hispec_verify_intermediate", "hispec_verify_target",
            "hispec_prefill", "hispec_device_status", "hispec_launch_count", "hispec_strerror",
            "hispec_profile_enable", "hispec_profile_read", "hispec_last_error", "hispec_exit_argmax_noalloc",
-           "hispec_debug_trace"]
+           "hispec_debug_trace", "hispec_accept_rejection", "hispec_sample"]
 
 
 class ModelDesc(ctypes.Structure):
@@ -61,7 +61,7 @@ class CHidden(ctypes.Structure):
 
 class CResult(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("n_accepted", "next_token", "argmax_ids", "top2", "logits", "hidden_out",
-                                               "tentative", "pending")]
+                                               "tentative", "pending")] + [("defer_accept", ctypes.c_int32)]
 
 
 _lib = None
@@ -96,6 +96,10 @@ def load() -> ctypes.CDLL:
         lib.hispec_last_error.restype = ctypes.c_char_p
         lib.hispec_exit_argmax_noalloc.argtypes = [vp, vp, vp, ctypes.c_float, i32, i32, vp, i32, vp, vp]
         lib.hispec_exit_argmax_noalloc.restype = ctypes.c_int
+        lib.hispec_accept_rejection.argtypes = [vp, vp, i32, vp, vp, i32, vp, i32, i32, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+        lib.hispec_accept_rejection.restype = ctypes.c_int
+        lib.hispec_sample.argtypes = [vp, vp, i32, vp, ctypes.c_int64, vp, ctypes.c_float, vp, i32]
+        lib.hispec_sample.restype = ctypes.c_int
         for name in EXPORTS[:7] + EXPORTS[9:11]:
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
@@ -152,10 +156,12 @@ class Result:
     hidden_out: Optional[torch.Tensor] = None
     tentative: Optional[torch.Tensor] = None
     pending: Optional[torch.Tensor] = None
+    defer_accept: bool = False
 
     def c(self) -> CResult:
         return CResult(_ptr(self.n_accepted), _ptr(self.next_token), _ptr(self.argmax_ids), _ptr(self.top2),
-                       _ptr(self.logits), _ptr(self.hidden_out), _ptr(self.tentative), _ptr(self.pending))
+                       _ptr(self.logits), _ptr(self.hidden_out), _ptr(self.tentative), _ptr(self.pending),
+                       1 if self.defer_accept else 0)
 
 
 class Context:
@@ -269,6 +275,28 @@ class Context:
                       n_rows: Optional[torch.Tensor], res: Result, stream=None, k: Optional[int] = None):
         self._verify(self.lib.hispec_verify_target, "hispec_verify_target", st, self.exits.L_i, self.exits.L_f,
                      draft_tokens, n_draft, n_rows, res, stream, k)
+
+    def accept_rejection(self, stage: int, st: KVState, draft_tokens: torch.Tensor, k: int, p_logits, q_logits,
+                         u_accept: torch.Tensor, u_sample: torch.Tensor, res: Result, stage_logits=None,
+                         temperature: float = 1.0, stream=None):
+        """Rejection-sampling acceptance for a verify call that ran with res.defer_accept (stage 1 =
+        intermediate, 2 = target); p_logits / q_logits [batch][max_rows][vocab] fp32 tensors or raw addresses."""
+        batch, stride = draft_tokens.shape
+        pp = p_logits if isinstance(p_logits, int) else _ptr(p_logits)
+        qp = q_logits if isinstance(q_logits, int) else _ptr(q_logits)
+        _check(self.lib.hispec_accept_rejection(self.handle, self._stream(stream), stage, ctypes.byref(self.exits),
+                                                ctypes.byref(st.c_kv()), batch, _ptr(draft_tokens), stride, k, pp, qp,
+                                                _ptr(u_accept), _ptr(u_sample), temperature, _ptr(stage_logits),
+                                                ctypes.byref(res.c())), "hispec_accept_rejection")
+
+    def sample(self, logits, row_stride: int, u, out_tokens, batch: int, out_stride: int = 1,
+               temperature: float = 1.0, stream=None):
+        """One token per sequence from softmax(logits row / temperature) by inversion with u[b]."""
+        lp = logits if isinstance(logits, int) else _ptr(logits)
+        up = u if isinstance(u, int) else _ptr(u)
+        op = out_tokens if isinstance(out_tokens, int) else _ptr(out_tokens)
+        _check(self.lib.hispec_sample(self.handle, self._stream(stream), batch, lp, row_stride, up, temperature, op,
+                                      out_stride), "hispec_sample")
 
     def prefill(self, st: KVState, tokens: torch.Tensor, n_tokens: torch.Tensor, first_token: torch.Tensor, stream=None):
         batch, max_tokens = tokens.shape

@@ -14,6 +14,7 @@
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
 #include "mega.cuh"
+#include "sampling.cuh"
 
 using namespace hispec;
 
@@ -430,6 +431,44 @@ extern "C" int hispec_debug_trace(hispec_ctx *c, unsigned long long *out, int ca
 
 extern "C" int64_t hispec_launch_count(const hispec_ctx *c) { return c ? c->launches : 0; }
 
+extern "C" int hispec_accept_rejection(hispec_ctx *c, void *stream, int stage, const hispec_exits *ex, const hispec_kv *kv,
+                                       int batch, const int32_t *draft_tokens, int token_stride, int k, const float *p_logits,
+                                       const float *q_logits, const float *u_accept, const float *u_sample,
+                                       float temperature, float *stage_logits, const hispec_result *res) {
+    if (!c || !ex || !kv || !draft_tokens || !p_logits || !q_logits || !u_accept || !u_sample) return HISPEC_EINVAL;
+    if ((stage != 1 && stage != 2) || batch < 1 || batch > c->d.max_batch || k < 1 || k + 1 > c->d.max_rows_per_seq)
+        return HISPEC_EINVAL;
+    if (!(0 < ex->L_d && ex->L_d < ex->L_i && ex->L_i < ex->L_f && ex->L_f <= c->d.n_layers)) return HISPEC_EINVAL;
+    if (!(temperature > 0.f) || token_stride < 1 || !kv->len_draft || !kv->len_inter || !kv->len_target) return HISPEC_EINVAL;
+    RejectArgs r;
+    memset(&r, 0, sizeof(r));
+    r.stage = stage; r.L_d = ex->L_d; r.L_i = ex->L_i; r.L_f = ex->L_f; r.k = k;
+    r.max_rows = c->d.max_rows_per_seq; r.vocab = c->d.vocab; r.token_stride = token_stride;
+    r.len_d = kv->len_draft; r.len_i = kv->len_inter; r.len_f = kv->len_target;
+    r.draft_tokens = draft_tokens; r.p_logits = p_logits; r.q_logits = q_logits;
+    r.u_accept = u_accept; r.u_sample = u_sample; r.inv_t = 1.0f / temperature; r.stage_logits = stage_logits;
+    if (res) { r.n_accepted = res->n_accepted; r.next_token = res->next_token; r.tentative = res->tentative; r.pending = res->pending; }
+    r.status = c->status;
+    // plain launch: the kernel must not start before the deferred verify call has finished
+    rejection_accept_kernel<<<batch, kSampleThreads, 0, (cudaStream_t)stream>>>(r);
+    c->launches++;
+    CK(cudaGetLastError());
+    return HISPEC_OK;
+}
+
+extern "C" int hispec_sample(hispec_ctx *c, void *stream, int batch, const float *logits, int64_t row_stride, const float *u,
+                             float temperature, int32_t *out_tokens, int out_stride) {
+    if (!c || !logits || !u || !out_tokens || batch < 1 || row_stride < c->d.vocab || !(temperature > 0.f) || out_stride < 1)
+        return HISPEC_EINVAL;
+    SampleArgs s;
+    s.logits = logits; s.row_stride = row_stride; s.u = u; s.inv_t = 1.0f / temperature; s.vocab = c->d.vocab;
+    s.out_tokens = out_tokens; s.out_stride = out_stride;
+    sample_kernel<<<batch, kSampleThreads, 0, (cudaStream_t)stream>>>(s);
+    c->launches++;
+    CK(cudaGetLastError());
+    return HISPEC_OK;
+}
+
 extern "C" int hispec_device_status(hispec_ctx *c, void *stream, uint32_t *host_out) {
     if (!c || !host_out) return HISPEC_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
@@ -663,6 +702,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         m.r.n_accepted = sc.res->n_accepted; m.r.next_token = sc.res->next_token;
         m.r.argmax_ids = sc.res->argmax_ids; m.r.top2 = sc.res->top2; m.r.tentative = sc.res->tentative;
         m.r.pending = sc.res->pending;
+        m.r.defer = sc.res->defer_accept;
         m.logits = sc.res->logits;
     }
     m.r.out_tokens = sc.out_tokens; m.r.n_tokens = sc.n_tokens;
@@ -809,6 +849,7 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         r.n_accepted = sc.res->n_accepted; r.next_token = sc.res->next_token;
         r.argmax_ids = sc.res->argmax_ids; r.top2 = sc.res->top2; r.tentative = sc.res->tentative;
         r.pending = sc.res->pending;
+        r.defer = sc.res->defer_accept;
     }
     r.out_tokens = sc.out_tokens;
     r.n_tokens = sc.n_tokens;

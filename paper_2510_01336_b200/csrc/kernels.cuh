@@ -343,6 +343,7 @@ struct AcceptArgs {
     int32_t *n_accepted, *next_token, *argmax_ids, *out_tokens, *tentative, *pending;
     float *top2;
     const int32_t *n_tokens;  // prefill: out_tokens only from the chunk that holds the last prompt token
+    int defer;                // verify calls: leave acceptance, lengths, V and the pending token to a later call
 };
 __global__ void head_reduce_accept_kernel(StageArgs a, RowMeta rm, const float *top_part, int n_tiles,
                                           int T_pad_total, AcceptArgs r, int32_t *argmax_ws) {
@@ -379,6 +380,7 @@ __global__ void head_reduce_accept_kernel(StageArgs a, RowMeta rm, const float *
     __syncthreads();
     if (threadIdx.x != 0) return;
     int p0 = rm.p0[b];
+    if (a.mode == 1 && r.defer) return;
     if (a.mode == 1) {
         int nd = rm.n_draft[b], acc = 0;
         while (acc < nd && acc < nr && r.draft_tokens[(size_t)b * r.token_stride + acc] == argmax_ws[b * a.R_pad + acc])

@@ -1173,6 +1173,7 @@ __device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b) {
     worker_bar();
     if (threadIdx.x != kMegaLeader) return;
     const int p0 = sh.p0[b];
+    if (a.mode == 1 && r.defer) return;
     if (a.mode == 1) {
         const int nd = sh.nd[b];
         int acc = 0;
