@@ -226,7 +226,7 @@ def extras(shape, w, args):
     draft exit scaled by 0.05, so that the exits agree as trained early-exit checkpoints do)."""
     import torch
     from paper_2510_01336_b200 import binding, workload as wl
-    from paper_2510_01336_b200.driver import ARLoop, HiSpecLoop, SelfSpecLoop
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecLoop, HiSpecSamplingLoop, SelfSpecLoop
     out = {}
     max_rows = ROUNDS * (N_D + 1) + 1
     max_pages = (N_PROMPT + 1024 + 15) // 16
@@ -266,6 +266,11 @@ def extras(shape, w, args):
     tps, toks, stats = timed_tokens(lambda c, s: HiSpecLoop(c, s, 1, N_D, ROUNDS), run_hs, wg)
     ss = timed_tokens(lambda c, s: SelfSpecLoop(c, s, 1, N_D), run_ss, wg)
     ar = timed_tokens(lambda c, s: ARLoop(c, s, 1), run_ar, wg)[0]
+    # the same loop with rejection-sampling acceptance at both stages (App. G), temperature 1
+    uni = lambda sr: wl.make_uniforms(shape, sr, 1, ROUNDS, N_D, max_rows)
+    rs = timed_tokens(lambda c, s: HiSpecSamplingLoop(c, s, 1, N_D, ROUNDS, uni), run_hs, wg)
+    out["rejection_sampling_gamma0.05"] = {"hispec_tokens_per_s": round(rs[0], 1), "tokens_per_super_round": round(rs[1] / 12, 2),
+                                           "over_greedy_hispec": round(rs[0] / tps, 2)}
     out["acceptance_shaped_gamma0.05"] = {"hispec_tokens_per_s": round(tps, 1), "tokens_per_super_round": round(toks / 12, 2),
                                           "selfspec_alg1_tokens_per_s": round(ss[0], 1), "tokens_per_alg1_round": round(ss[1] / 16, 2),
                                           "ar_tokens_per_s": round(ar, 1), "hispec_over_ar": round(tps / ar, 2),

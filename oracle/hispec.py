@@ -523,6 +523,62 @@ class HiSpecOracle:
         stats.committed = min(len(x) - n0, n_gen)
         return x[n0: n0 + n_gen]
 
+    def hispec_generate_sampling(self, prompt: Sequence[int], n_gen: int, N_d: int, rounds: int,
+                                 uniforms: Callable[[int], dict], temperature: float = 1.0, seq: int = 0,
+                                 stats: Optional[GenStats] = None) -> List[int]:
+        """Algorithm 2 with the rejection-sampling rule of App. G at both verification stages: drafts are
+        drawn from p_{L_d}, the intermediate stage filters them into V (distributed as p_{L_i}), the target
+        stage filters V (result distributed as p_{L_f}).  Fixed `rounds` per target verification, bonus row at
+        the intermediate stage.  `uniforms(super_round)` returns the arrays documented in the workload
+        generator (`draft`, `acc_i`, `smp_i`, `acc_t`, `smp_t`); `seq` selects the batch column.  The first
+        generated token is the prefill's greedy token."""
+        from . import rejection as rj
+        stats = stats if stats is not None else GenStats()
+        cap_rows = rounds * (N_d + 1) + 2
+        st = self.new_state(len(prompt) + n_gen + cap_rows + 2, cap_rows)
+        pending = self.prefill(st, prompt).argmax_ids[0]
+        x = [int(t) for t in prompt] + [pending]
+        n0, sr = len(prompt), 0
+        while len(x) - n0 < n_gen:
+            U = {k: np.asarray(v) for k, v in uniforms(sr).items()}
+            sr += 1
+            V: List[int] = []
+            PV: List[np.ndarray] = []
+            for r in range(rounds):
+                S, P_rows, u = [], [], pending
+                for j in range(N_d + 1):
+                    o = self.draft_step(st, u)
+                    stats.draft_steps += 1
+                    if j < N_d:
+                        p = rj.softmax_f32(o.logits[0], temperature)
+                        u = rj.sample_inverse_cdf(p, float(U["draft"][r, j, seq]))
+                        S.append(u)
+                        P_rows.append(p)
+                R = N_d + 1
+                p0 = st.len_i
+                out = self.verify_intermediate(st, S, R)       # rows, KV, exit rows; its greedy decision is replaced below
+                Q = rj.softmax_f32(out.logits[:R], temperature)
+                res, a = rj.rejection_verify(S, np.stack(P_rows), Q, U["acc_i"][r, seq], float(U["smp_i"][r, seq]))
+                st.len_d = st.len_i = p0 + min(a + 1, R)
+                V += res
+                PV += [Q[j] for j in range(len(res))]
+                pending = res[-1]
+                stats.inter_calls += 1
+                stats.inter_accepted += a
+            R = len(V)
+            p0 = st.len_f
+            out = self.verify_target(st, V, R)
+            Qf = rj.softmax_f32(out.logits[:R], temperature)
+            F, a = rj.rejection_verify(V, np.stack(PV), Qf, U["acc_t"][seq], float(U["smp_t"][seq]))
+            st.len_d = st.len_i = st.len_f = p0 + min(a + 1, R)
+            x += F
+            pending = F[-1]
+            stats.target_calls += 1
+            stats.target_checked += len(V)
+            stats.target_accepted += a
+        stats.committed = min(len(x) - n0, n_gen)
+        return x[n0: n0 + n_gen]
+
     def _generate_observed(self, st, pending, N_d, bonus, stats, draft_override, observer, ctx_tokens):
         S, u = [], pending
         for j in range(N_d + (1 if bonus else 0)):

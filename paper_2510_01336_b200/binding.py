@@ -117,8 +117,8 @@ def _check(rc: int, what: str):
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
-    if t is None:
-        return None
+    if t is None or isinstance(t, int):   # an int is a raw device address (a row inside a larger buffer)
+        return t
     assert t.is_cuda and t.is_contiguous()
     return t.data_ptr()
 

@@ -102,6 +102,7 @@ struct hispec_ctx_ext {
     int n_mega_heads;
     const float **d_attn_norm, **d_ffn_norm;  // device arrays of device pointers
     float *ssq;                // [T_alloc][ceil(d / 128)] chunk sums of squares
+    float *rs_stats, *rs_dec, *rs_wsum;   // workspace of the sampling kernels (chunk statistics, decisions, chunk weights)
     float2 *rope;              // [T_alloc][head_dim / 2] (cos, sin) of this call's rows, filled by the persistent kernel
     unsigned *bar;             // grid barrier counters, used alternately by successive launches
     int bar_sel;
@@ -327,6 +328,12 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     ok = ok && alloc((void **)&c->ext.d_ffn_norm, sizeof(float *) * L);
     ok = ok && alloc((void **)&c->ext.ssq, sizeof(float) * (size_t)T_alloc * ceil_div(d.d_model, kSsqChunk));
     ok = ok && alloc((void **)&c->ext.rope, sizeof(float2) * (size_t)T_alloc * (d.head_dim / 2));
+    {
+        const size_t chunks = ceil_div(d.vocab, kVChunk);
+        ok = ok && alloc((void **)&c->ext.rs_stats, sizeof(float) * 2 * 2 * chunks * (size_t)d.max_batch * d.max_rows_per_seq);
+        ok = ok && alloc((void **)&c->ext.rs_dec, sizeof(float) * kDecFloats * (size_t)d.max_batch);
+        ok = ok && alloc((void **)&c->ext.rs_wsum, sizeof(float) * 2 * chunks * (size_t)d.max_batch);
+    }
     ok = ok && alloc((void **)&c->ext.bar, 2 * sizeof(unsigned));
     if (env_int("HISPEC_TRACE", 0)) ok = ok && alloc((void **)&c->ext.trace, 1024 * sizeof(unsigned long long));
     if (!ok) { hispec_destroy(c); return HISPEC_ENOMEM; }
@@ -381,7 +388,7 @@ extern "C" int hispec_destroy(hispec_ctx *c0) {
     hispec_ctx_full *c = static_cast<hispec_ctx_full *>(c0);
     void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->attn_part, c->top_part, c->logits_ws, c->inv_freq,
                     c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status,
-                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace, c->ext.rope};
+                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace, c->ext.rope, c->ext.rs_stats, c->ext.rs_dec, c->ext.rs_wsum};
     for (void *p : bufs)
         if (p) cudaFree(p);
     delete[] c->wqkv; delete[] c->wo; delete[] c->wgu; delete[] c->wdown; delete[] c->attn_norm; delete[] c->ffn_norm;
@@ -431,6 +438,22 @@ extern "C" int hispec_debug_trace(hispec_ctx *c, unsigned long long *out, int ca
 
 extern "C" int64_t hispec_launch_count(const hispec_ctx *c) { return c ? c->launches : 0; }
 
+// the four sampling kernels, in order, as plain launches (each must see the previous one's results and, first of
+// all, those of the deferred verify call)
+static int run_sampling(hispec_ctx *c, cudaStream_t st, RsArgs &r, int batch) {
+    hispec_ctx_ext *x = ext_of(c);
+    r.chunks = ceil_div(r.vocab, kVChunk);
+    r.ws_stats = x->rs_stats; r.ws_dec = x->rs_dec; r.ws_wsum = x->rs_wsum;
+    r.status = c->status;
+    rs_stats_kernel<<<dim3(r.chunks, batch * r.rows_per_seq, 2), kRsThreads, 0, st>>>(r);
+    rs_decide_kernel<<<batch, 256, 0, st>>>(r, batch);
+    rs_weight_kernel<<<dim3(r.chunks, batch), kRsThreads, 0, st>>>(r);
+    rs_pick_kernel<<<batch, kRsThreads, 0, st>>>(r);
+    c->launches += 4;
+    CK(cudaGetLastError());
+    return HISPEC_OK;
+}
+
 extern "C" int hispec_accept_rejection(hispec_ctx *c, void *stream, int stage, const hispec_exits *ex, const hispec_kv *kv,
                                        int batch, const int32_t *draft_tokens, int token_stride, int k, const float *p_logits,
                                        const float *q_logits, const float *u_accept, const float *u_sample,
@@ -440,33 +463,30 @@ extern "C" int hispec_accept_rejection(hispec_ctx *c, void *stream, int stage, c
         return HISPEC_EINVAL;
     if (!(0 < ex->L_d && ex->L_d < ex->L_i && ex->L_i < ex->L_f && ex->L_f <= c->d.n_layers)) return HISPEC_EINVAL;
     if (!(temperature > 0.f) || token_stride < 1 || !kv->len_draft || !kv->len_inter || !kv->len_target) return HISPEC_EINVAL;
-    RejectArgs r;
+    RsArgs r;
     memset(&r, 0, sizeof(r));
     r.stage = stage; r.L_d = ex->L_d; r.L_i = ex->L_i; r.L_f = ex->L_f; r.k = k;
     r.max_rows = c->d.max_rows_per_seq; r.vocab = c->d.vocab; r.token_stride = token_stride;
+    r.rows_per_seq = k + 1;
+    r.p_seq_stride = r.q_seq_stride = (long long)c->d.max_rows_per_seq * c->d.vocab;
     r.len_d = kv->len_draft; r.len_i = kv->len_inter; r.len_f = kv->len_target;
     r.draft_tokens = draft_tokens; r.p_logits = p_logits; r.q_logits = q_logits;
     r.u_accept = u_accept; r.u_sample = u_sample; r.inv_t = 1.0f / temperature; r.stage_logits = stage_logits;
     if (res) { r.n_accepted = res->n_accepted; r.next_token = res->next_token; r.tentative = res->tentative; r.pending = res->pending; }
-    r.status = c->status;
-    // plain launch: the kernel must not start before the deferred verify call has finished
-    rejection_accept_kernel<<<batch, kSampleThreads, 0, (cudaStream_t)stream>>>(r);
-    c->launches++;
-    CK(cudaGetLastError());
-    return HISPEC_OK;
+    return run_sampling(c, (cudaStream_t)stream, r, batch);
 }
 
 extern "C" int hispec_sample(hispec_ctx *c, void *stream, int batch, const float *logits, int64_t row_stride, const float *u,
                              float temperature, int32_t *out_tokens, int out_stride) {
-    if (!c || !logits || !u || !out_tokens || batch < 1 || row_stride < c->d.vocab || !(temperature > 0.f) || out_stride < 1)
+    if (!c || !logits || !u || !out_tokens || batch < 1 || batch > c->d.max_batch || row_stride < c->d.vocab ||
+        !(temperature > 0.f) || out_stride < 1)
         return HISPEC_EINVAL;
-    SampleArgs s;
-    s.logits = logits; s.row_stride = row_stride; s.u = u; s.inv_t = 1.0f / temperature; s.vocab = c->d.vocab;
-    s.out_tokens = out_tokens; s.out_stride = out_stride;
-    sample_kernel<<<batch, kSampleThreads, 0, (cudaStream_t)stream>>>(s);
-    c->launches++;
-    CK(cudaGetLastError());
-    return HISPEC_OK;
+    RsArgs r;
+    memset(&r, 0, sizeof(r));
+    r.stage = 0; r.k = 0; r.max_rows = c->d.max_rows_per_seq; r.vocab = c->d.vocab; r.rows_per_seq = 1;
+    r.q_seq_stride = row_stride; r.q_logits = logits; r.u_sample = u; r.inv_t = 1.0f / temperature;
+    r.out_tokens = out_tokens; r.out_stride = out_stride;
+    return run_sampling(c, (cudaStream_t)stream, r, batch);
 }
 
 extern "C" int hispec_device_status(hispec_ctx *c, void *stream, uint32_t *host_out) {

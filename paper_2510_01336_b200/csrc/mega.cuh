@@ -1088,6 +1088,21 @@ __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, 
     return true;
 }
 
+// optional output of the exit head: logits of eight rows (columns c0..c0+7 of the accumulators) for this thread's
+// vocabulary entry; 1 / rms of the rows is taken once per warp.  Kept out of line: the hot path never runs it.
+struct Float8 { float a, b, c, d, e, f, g, h; };   // passed by value: in registers
+__device__ __noinline__ void mega_store_logits(const MegaArgs &m, MegaShared &sh, int N, int n, int c0, Float8 s, int lane) {
+    const float v[8] = {s.a, s.b, s.c, s.d, s.e, s.f, s.g, s.h};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int t = c0 + i;
+        if (t >= m.T_pad) break;
+        const float inv = mega_inv_rms_warp(m, t, lane);
+        const int b = t / m.a.R_pad, j = t % m.a.R_pad;
+        if (n < N && j < sh.nr[b]) m.logits[((size_t)b * m.a.max_rows + j) * N + n] = v[i] * inv;
+    }
+}
+
 // warps 4..7, exit head: each tile's accumulator is the sum of the two pipelines' K halves; every
 // column (activation row) is reduced to its top-2 over this warp's 32 vocabulary entries
 __device__ __forceinline__ bool mega_epilogue_head(const MegaGemm *g, const MegaArgs &m, MegaShared &sh,
@@ -1112,15 +1127,14 @@ __device__ __forceinline__ bool mega_epilogue_head(const MegaGemm *g, const Mega
             float v[8], w[8];
             mega_acc_ld8(taddr[0], c0, m.t_box, m.planes, v);
             mega_acc_ld8(taddr[1], c0, m.t_box, m.planes, w);
+            if (m.logits)   // parity / sampling output: off the hot path
+                mega_store_logits(m, sh, g->N, n, c0, Float8{v[0] + w[0], v[1] + w[1], v[2] + w[2], v[3] + w[3], v[4] + w[4], v[5] + w[5],
+                                                             v[6] + w[6], v[7] + w[7]}, lane);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 if (c0 + i >= m.T_pad) break;
                 const int t = c0 + i;
                 const float val = (n < g->N) ? v[i] + w[i] : -INFINITY;
-                if (m.logits && n < g->N) {
-                    const int b = t / m.a.R_pad, j = t % m.a.R_pad;
-                    if (j < sh.nr[b]) m.logits[((size_t)b * m.a.max_rows + j) * g->N + n] = val * mega_inv_rms(m, t);
-                }
                 Top2 best = top2_warp(Top2{val, -INFINITY, n < g->N ? n : 0x7fffffff});
                 if (lane == 0) {
                     float *o = m.top_part + ((size_t)(tile * 4 + lg) * m.T_pad + t) * 4;

@@ -267,6 +267,79 @@ class HiSpecAdaptiveLoop(HiSpecDynamicLoop):
         return new
 
 
+class HiSpecSamplingLoop(HiSpecLoop):
+    """Algorithm 2 with rejection-sampling acceptance at both stages (App. G): draft tokens are sampled
+    from the draft exit, every verify call runs with deferred acceptance and writes its logits, and
+    hispec_accept_rejection decides on the device.  A super-round is still enqueued without a host
+    synchronisation; the uniforms it consumes are inputs (`uniforms(super_round) -> dict`, see
+    workload.make_uniforms).  `on_accept(stage, round, record)` -- testing aid -- is called after every
+    acceptance with copies of everything it read and wrote (this synchronises)."""
+
+    def __init__(self, ctx, st, batch, N_d, rounds, uniforms: Callable[[int], dict], temperature: float = 1.0,
+                 on_accept: Optional[Callable] = None, device="cuda"):
+        super().__init__(ctx, st, batch, N_d, rounds, bonus_inter=True, device=device)
+        V, R = ctx.shape.vocab, ctx.max_rows
+        f = lambda: torch.zeros((batch, R, V), dtype=torch.float32, device=device)
+        self.logits_d, self.logits_i, self.logits_t, self.logits_stage = f(), f(), f(), f()
+        i32 = lambda *sh: torch.zeros(sh, dtype=torch.int32, device=device)
+        # a draft step writes its logits to row 0 of the buffer it is given: step j gets the buffer shifted by j rows
+        self.res_d = [binding.Result(i32(batch), i32(batch), logits=self.logits_d.data_ptr() + 4 * j * V) for j in range(N_d)]
+        for r in self.res_i:
+            r.logits, r.defer_accept = self.logits_i, True
+        self.res_t.logits, self.res_t.defer_accept = self.logits_t, True
+        self.uniforms, self.temperature, self.on_accept = uniforms, temperature, on_accept
+        self.sr = 0
+
+    def _record(self, stage, rnd, S, k, p, q, ua, us, res, lens_before):
+        if self.on_accept is None:
+            return
+        torch.cuda.synchronize()
+        st = self.st
+        self.on_accept(stage, rnd, {
+            "S": S.cpu().clone(), "k": k, "p": p.cpu().clone(), "q": q.cpu().clone(), "u_acc": ua.cpu().clone(),
+            "u_smp": us.cpu().clone(), "n_accepted": res.n_accepted.cpu().clone(), "next_token": res.next_token.cpu().clone(),
+            "lens_before": lens_before,
+            "lens_after": (st.len_draft.cpu().clone(), st.len_inter.cpu().clone(), st.len_target.cpu().clone()),
+            "V": self.V.cpu().clone(), "pending": self.pending.cpu().clone()})
+
+    def _lens(self):
+        if self.on_accept is None:
+            return None
+        torch.cuda.synchronize()
+        st = self.st
+        return (st.len_draft.cpu().clone(), st.len_inter.cpu().clone(), st.len_target.cpu().clone())
+
+    def enqueue_super_round(self, stream=None):
+        ctx, st, N_d, B, T = self.ctx, self.st, self.N_d, self.B, self.temperature
+        Vc, R = ctx.shape.vocab, ctx.max_rows
+        U = {k: v.cuda(non_blocking=True) for k, v in self.uniforms(self.sr).items()}
+        self.sr += 1
+        S_ptr = self.S.data_ptr()
+        for r in range(self.rounds):
+            for j in range(N_d):
+                if j == 0:
+                    ctx.draft(st, self.pending, None, res=self.res_d[j], batch=B, in_stride=1, stream=stream)
+                else:
+                    ctx.draft(st, S_ptr + 4 * (j - 1), None, res=self.res_d[j], batch=B, in_stride=N_d, stream=stream)
+                ctx.sample(self.logits_d.data_ptr() + 4 * j * Vc, R * Vc, U["draft"][r, j], S_ptr + 4 * j, B,
+                           out_stride=N_d, temperature=T, stream=stream)
+            ctx.draft(st, S_ptr + 4 * (N_d - 1), None, batch=B, in_stride=N_d, stream=stream)
+            ctx.verify_intermediate(st, self.S, None, None, self.res_i[r], stream=stream, k=N_d)
+            lens = self._lens()
+            ctx.accept_rejection(1, st, self.S, N_d, self.logits_d, self.logits_i, U["acc_i"][r], U["smp_i"][r],
+                                 self.res_i[r], stage_logits=self.logits_stage, temperature=T, stream=stream)
+            self._record(1, r, self.S, N_d, self.logits_d, self.logits_i, U["acc_i"][r], U["smp_i"][r], self.res_i[r], lens)
+            self.stats.draft_steps += N_d + 1
+            self.stats.inter_calls += 1
+        ctx.verify_target(st, self.V, None, None, self.res_t, stream=stream, k=R - 1)
+        lens = self._lens()
+        ctx.accept_rejection(2, st, self.V, R - 1, self.logits_stage, self.logits_t, U["acc_t"], U["smp_t"], self.res_t,
+                             temperature=T, stream=stream)
+        self._record(2, 0, self.V, R - 1, self.logits_stage, self.logits_t, U["acc_t"], U["smp_t"], self.res_t, lens)
+        self.stats.target_calls += 1
+        self.stats.super_rounds += 1
+
+
 class SelfSpecLoop:
     """Algorithm 1 (single-stage self-speculation): N_d (+1) draft steps at L_d, then one verification of the
     block by the final layer -- hispec_verify_intermediate over [L_d, L_f) with the L_f exit."""

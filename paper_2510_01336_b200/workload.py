@@ -171,6 +171,18 @@ def make_tokens(shape: ModelShape, n: int, seed_offset: int = 1000) -> torch.Ten
     return torch.randint(0, shape.vocab, (n,), generator=g, dtype=torch.int64).to(torch.int32)
 
 
+def make_uniforms(shape: ModelShape, super_round: int, batch: int, rounds: int, n_draft: int, max_rows: int,
+                  seed_offset: int = 5000) -> dict:
+    """The uniform random numbers one super-round of sampling-based decoding consumes (fp32, CPU, in [0,1)):
+    `draft` [rounds][n_draft][batch] (one per sampled draft token), `acc_i` [rounds][batch][max_rows] and
+    `smp_i` [rounds][batch] (accept tests and the replacement / bonus draw of each intermediate verification),
+    `acc_t` [batch][max_rows] and `smp_t` [batch] (the same for the target verification)."""
+    g = torch.Generator().manual_seed(shape.seed + seed_offset + 7919 * super_round)
+    r = lambda *sh: torch.rand(sh, generator=g, dtype=torch.float32)
+    return {"draft": r(rounds, n_draft, batch), "acc_i": r(rounds, batch, max_rows), "smp_i": r(rounds, batch),
+            "acc_t": r(batch, max_rows), "smp_t": r(batch)}
+
+
 def make_prompt_lengths(shape: ModelShape, batch: int, lo: int, hi: int, seed_offset: int = 2000) -> List[int]:
     """Per-sequence prompt lengths i.i.d. uniform integers in [lo, hi]."""
     g = torch.Generator().manual_seed(shape.seed + seed_offset)

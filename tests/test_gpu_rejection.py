@@ -140,3 +140,77 @@ def test_inversion_sampling_matches_oracle():
             assert _token_ok(P[s], float(u[s]), int(out[s, 0])), (temp, s)
         assert int(out[2, 0]) < 5 and torch.all(out[:, 1] == -1)
     ctx.close()
+
+
+def test_sampling_loop_end_to_end():
+    """The sampling decoding loop on the device: (1) every acceptance the loop makes is re-derived by the
+    oracle from the very logits, drafts and uniforms the kernel read; (2) at a temperature close to zero the
+    loop reproduces the GPU's own greedy auto-regressive output (the limit in which sampling is greedy)."""
+    b = _binding()
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecSamplingLoop
+    shape = wl.TINY
+    scale = {l: 0.05 for l in range(shape.L_d, shape.L_f)}
+    wg = wl.make_weights(shape, resid_scale=scale).to("cuda")
+    B, N_d, rounds, n_prompt, n_gen = 2, 3, 2, 48, 20
+    max_rows = rounds * (N_d + 1) + 3
+    max_pages = (n_prompt + n_gen + 40) // 16 + 1
+    prompts = [wl.make_tokens(shape, n_prompt, seed_offset=1000 + s).tolist() for s in range(B)]
+    bt = wl.make_block_table(shape, B, max_pages)
+    uni = lambda sr: wl.make_uniforms(shape, sr, B, rounds, N_d, max_rows)
+
+    records = []
+    ctx = b.Context(shape, wg, max_batch=B, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    st = ctx.new_state(B, max_pages * B, bt)
+    loop = HiSpecSamplingLoop(ctx, st, B, N_d, rounds, uni, temperature=1.0,
+                              on_accept=lambda stage, rnd, rec: records.append((stage, rnd, rec)))
+    loop.prefill(prompts)
+    toks = loop.generate(n_gen)
+    assert ctx.status() == 0
+    assert all(len(t) == n_gen and all(0 <= x < shape.vocab for x in t) for t in toks)
+    compared = kept = 0
+    for stage, rnd, rec in records:
+        P = rj.softmax_f32(rec["p"].numpy())
+        Q = rj.softmax_f32(rec["q"].numpy())
+        ld, li, lf = (x.tolist() for x in rec["lens_before"])
+        for s in range(B):
+            avail = ld[s] - li[s] if stage == 1 else li[s] - lf[s]
+            nr = min(avail, rec["k"] + 1)
+            nd = min(nr, rec["k"])
+            assert nr >= 1
+            S = rec["S"][s, :nd].tolist()
+            out, a = rj.rejection_verify(S, P[s, :nd], Q[s, :nr], rec["u_acc"][s].tolist(), float(rec["u_smp"][s]))
+            fragile = False
+            for j in range(min(a + 1, nd)):
+                ratio = 1.0 if not P[s, j, S[j]] > 0 else min(1.0, float(Q[s, j, S[j]]) / float(P[s, j, S[j]]))
+                fragile |= abs(float(rec["u_acc"][s, j]) - ratio) < TOL_U and ratio < 1.0
+            if fragile:
+                continue
+            compared += 1
+            kept += a
+            assert int(rec["n_accepted"][s]) == a
+            p0 = li[s] if stage == 1 else lf[s]
+            nl = p0 + min(a + 1, nr)
+            la = [int(x[s]) for x in rec["lens_after"]]
+            assert la[0] == nl and la[1] == nl and la[2] == (nl if stage == 2 else lf[s])
+            if a < nr:
+                w = rj.residual(P[s, a] if a < nd else None, Q[s, a])
+                if not w.sum() > 0:
+                    w = Q[s, a]
+                nxt = int(rec["next_token"][s])
+                assert _token_ok(w, float(rec["u_smp"][s]), nxt) and int(rec["pending"][s]) == nxt
+            if stage == 1:
+                d0 = li[s] - lf[s]
+                assert rec["V"][s, d0:d0 + a].tolist() == S[:a]
+    assert compared >= 10 and kept > 0
+    ctx.close()
+
+    outs = {}
+    for name in ("ar", "cold"):
+        ctx = b.Context(shape, wg, max_batch=B, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+        st = ctx.new_state(B, max_pages * B, bt)
+        loop = ARLoop(ctx, st, B) if name == "ar" else HiSpecSamplingLoop(ctx, st, B, N_d, rounds, uni, temperature=1e-3)
+        loop.prefill(prompts)
+        outs[name] = loop.generate(n_gen)
+        assert ctx.status() == 0
+        ctx.close()
+    assert outs["cold"] == outs["ar"]

@@ -90,3 +90,25 @@ def test_two_stage_composition_reproduces_the_final_distribution():
     assert np.all(np.abs(counts / n - pf) < 4 * np.sqrt(pf * (1 - pf) / n) + 1e-3)
     m = second.sum()
     assert m > n / 4 and np.all(np.abs(second / m - pf) < 5 * np.sqrt(pf * (1 - pf) / m) + 2e-3)
+
+
+def test_sampling_generation_at_low_temperature_is_greedy_decoding():
+    """As the temperature goes to 0 every distribution becomes one-hot on its argmax: drafts are the greedy
+    drafts, the ratio test keeps exactly the tokens the verifier's argmax agrees with, the residual is the
+    verifier's argmax -- so sampling-based HiSpec must reproduce greedy auto-regressive decoding."""
+    from paper_2510_01336_b200 import workload as wl
+    from tests.helpers import oracle_for
+    shape = wl.TINY
+    scale = {l: 0.05 for l in range(shape.L_d, shape.L_f)}
+    _, _, hs = oracle_for(shape, resid_scale=scale)
+    prompt = wl.make_tokens(shape, 20).tolist()
+    n_gen, N_d, rounds = 24, 3, 2
+    uni = lambda sr: wl.make_uniforms(shape, sr, 1, rounds, N_d, rounds * (N_d + 1) + 2)
+    ar = hs.ar_generate(prompt, n_gen)
+    st = __import__("oracle.hispec", fromlist=["GenStats"]).GenStats()
+    out = hs.hispec_generate_sampling(prompt, n_gen, N_d, rounds, uni, temperature=1e-3, stats=st)
+    assert out == ar
+    assert st.inter_accepted > 0 and st.target_accepted > 0
+    # at temperature 1 the output differs from greedy (it is a sample) but every stage call keeps the state consistent
+    out1 = hs.hispec_generate_sampling(prompt, n_gen, N_d, rounds, uni, temperature=1.0)
+    assert len(out1) == n_gen and out1[0] == ar[0] and out1 != ar
