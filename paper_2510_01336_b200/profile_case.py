@@ -1,6 +1,6 @@
 """A small stand-alone case of the hot call for profilers: one intermediate-verification call
-(layers [L_d, L_i) + exit head) of the Llama-3-8B-shaped model on seeded random state, repeated a few
-times.  Device footprint ~5 GB (8 layers of weights + head + a 1024-token KV pool): large against the
+(layers [L_d, L_i) + exit head) of the Llama-3-8B-shaped model (or another shape, --shape) on seeded random
+state, repeated a few times.  Device footprint ~5 GB at the default shape (8 layers of weights + head + a 1024-token KV pool): large against the
 126 MB L2, small enough for a multi-pass ncu capture.
 
     python -m paper_2510_01336_b200.profile_case --calls 3
@@ -20,8 +20,10 @@ def main():
     ap.add_argument("--rows", type=int, default=6)
     ap.add_argument("--ctx", type=int, default=1024)
     ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--shape", default="llama3-8b-shape", choices=sorted(wl.SHAPES),
+                    help="model shape; the call covers its intermediate range [L_d, L_i)")
     args = ap.parse_args()
-    shape = wl.L3_8B
+    shape = wl.SHAPES[args.shape]
     layers = list(range(shape.L_d, shape.L_i))
     w = wl.make_weights(shape, layers=layers, device="cuda", with_emb=False)
     max_rows = 13
@@ -51,7 +53,8 @@ def main():
     by = len(layers) * shape.layer_weight_bytes + shape.head_bytes + len(layers) * shape.kv_bytes_per_token_layer * (args.ctx + args.rows)
     for i in range(args.calls):
         ms = ev[i].elapsed_time(ev[i + 1])
-        print(f"call {i}: {ms * 1e3:.1f} us, {by / ms / 1e6:.0f} GB/s algorithmic, status {status}")
+        print(f"{shape.name} [{shape.L_d},{shape.L_i}) rows {args.rows} ctx {args.ctx} call {i}: {ms * 1e3:.1f} us, "
+              f"{by / 1e9:.2f} GB, {by / ms / 1e6:.0f} GB/s algorithmic, status {status}")
     ctx.close()
 
 

@@ -65,10 +65,16 @@ L3_8B = ModelShape("llama3-8b-shape", 32, 4096, 32, 8, 128, 14336, 128256, 50000
                    L_d=8, L_i=16, L_f=32, seed=20251002)
 L2_13B = ModelShape("llama2-13b-shape", 40, 5120, 40, 40, 128, 13824, 32000, 10000.0,
                     L_d=10, L_i=20, L_f=40, seed=20251004)
+# The two larger models of the paper's tables, by layer shape (Table 1: CodeLlama-34B with exits 7/12/48,
+# Llama-2-70B with exits 10/20/80): GQA 8:1, d 8192.
+CL_34B = ModelShape("codellama-34b-shape", 48, 8192, 64, 8, 128, 22016, 32000, 1000000.0,
+                    L_d=7, L_i=12, L_f=48, seed=20251006)
+L2_70B = ModelShape("llama2-70b-shape", 80, 8192, 64, 8, 128, 28672, 32000, 10000.0,
+                    L_d=10, L_i=20, L_f=80, seed=20251007)
 # Small odd shapes for tests: GQA 2:1, K/M tails, head_dim 128.
 MINI_GQA = ModelShape("mini-gqa", 6, 320, 4, 2, 128, 400, 1000, 10000.0, L_d=2, L_i=3, L_f=6, seed=77)
 
-SHAPES = {s.name: s for s in (TINY, L3_8B, L2_13B, MINI_GQA)}
+SHAPES = {s.name: s for s in (TINY, L3_8B, L2_13B, CL_34B, L2_70B, MINI_GQA)}
 
 _KINDS = {"tok_emb": 1, "head": 2, "wqkv": 3, "wo": 4, "wgu": 5, "wdown": 6}
 

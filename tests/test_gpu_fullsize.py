@@ -101,6 +101,21 @@ def test_llama2_13b_shape_two_layers():
     _run_case(shape, 10, 12, "verify_i", [2048, 777], [7, 7], [6, 6], 7, seed_offset=4200)
 
 
+def test_codellama_34b_shape_two_layers():
+    """CodeLlama-34B layer shape (GQA 8:1, d 8192, ffn 22016): two layers of the intermediate range [7, 12),
+    batch 1, context 1024, k = 5 with the bonus row."""
+    import dataclasses
+    shape = dataclasses.replace(wl.CL_34B, L_d=7, L_i=9, L_f=48)
+    _run_case(shape, 7, 9, "verify_i", [1024], [6], [5], 7, seed_offset=4300)
+
+
+def test_llama2_70b_shape_two_layers():
+    """Llama-2-70B layer shape (GQA 8:1, d 8192, ffn 28672): two layers of the target range, batch 2, ragged."""
+    import dataclasses
+    shape = dataclasses.replace(wl.L2_70B, L_d=10, L_i=20, L_f=22)
+    _run_case(shape, 20, 22, "verify_t", [600, 1023], [9, 4], [9, 4], 10, seed_offset=4400)
+
+
 def test_llama3_8b_shape_plain_bf16_activations():
     """The same benchmarked call with plain bf16 tensor-core inputs (no hi/lo split): still inside the tolerances."""
     from paper_2510_01336_b200 import binding
