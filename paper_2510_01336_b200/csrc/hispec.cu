@@ -102,6 +102,7 @@ struct hispec_ctx_ext {
     int n_mega_heads;
     const float **d_attn_norm, **d_ffn_norm;  // device arrays of device pointers
     float *ssq;                // [T_alloc][ceil(d / 128)] chunk sums of squares
+    float *cta_top;            // [sm_count][T_alloc][4] per-CTA top-2 records of the persistent kernel
     float *rs_stats, *rs_dec, *rs_wsum;   // workspace of the sampling kernels (chunk statistics, decisions, chunk weights)
     float2 *rope;              // [T_alloc][head_dim / 2] (cos, sin) of this call's rows, filled by the persistent kernel
     unsigned *bar;             // grid barrier counters, used alternately by successive launches
@@ -328,6 +329,7 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     ok = ok && alloc((void **)&c->ext.d_ffn_norm, sizeof(float *) * L);
     ok = ok && alloc((void **)&c->ext.ssq, sizeof(float) * (size_t)T_alloc * ceil_div(d.d_model, kSsqChunk));
     ok = ok && alloc((void **)&c->ext.rope, sizeof(float2) * (size_t)T_alloc * (d.head_dim / 2));
+    ok = ok && alloc((void **)&c->ext.cta_top, sizeof(float) * 4 * (size_t)c->sm_count * T_alloc);
     {
         const size_t chunks = ceil_div(d.vocab, kVChunk);
         ok = ok && alloc((void **)&c->ext.rs_stats, sizeof(float) * 2 * 2 * chunks * (size_t)d.max_batch * d.max_rows_per_seq);
@@ -388,7 +390,7 @@ extern "C" int hispec_destroy(hispec_ctx *c0) {
     hispec_ctx_full *c = static_cast<hispec_ctx_full *>(c0);
     void *bufs[] = {c->x, c->act_d, c->act_o, c->act_f, c->q, c->part, c->attn_part, c->top_part, c->logits_ws, c->inv_freq,
                     c->rows.p0, c->rows.n_rows, c->rows.n_draft, c->rows.dst_row, c->argmax_ws, c->status,
-                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace, c->ext.rope, c->ext.rs_stats, c->ext.rs_dec, c->ext.rs_wsum};
+                    c->ext.d_gemms, c->ext.d_attn_norm, c->ext.d_ffn_norm, c->ext.ssq, c->ext.bar, c->ext.trace, c->ext.rope, c->ext.cta_top, c->ext.rs_stats, c->ext.rs_dec, c->ext.rs_wsum};
     for (void *p : bufs)
         if (p) cudaFree(p);
     delete[] c->wqkv; delete[] c->wo; delete[] c->wgu; delete[] c->wdown; delete[] c->attn_norm; delete[] c->ffn_norm;
@@ -699,7 +701,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     m.k_pages = (__nv_bfloat16 *)kv.k_pages; m.v_pages = (__nv_bfloat16 *)kv.v_pages;
     m.block_table = kv.block_table; m.n_pages = kv.n_pages; m.first_layer = kv.first_layer;
     m.x = c->x; m.act_d = c->act_d; m.act_o = c->act_o; m.act_f = c->act_f; m.q = c->q; m.part = c->part;
-    m.attn_part = c->attn_part; m.top_part = c->top_part; m.ssq = x->ssq; m.inv_freq = c->inv_freq; m.rope = x->rope;
+    m.attn_part = c->attn_part; m.top_part = c->top_part; m.ssq = x->ssq; m.inv_freq = c->inv_freq; m.rope = x->rope; m.cta_top = x->cta_top;
     m.G = d.n_q_heads / d.n_kv_heads;
     const int QR = m.G * a.R_pad;
     m.n_mg = ceil_div(QR, 64);

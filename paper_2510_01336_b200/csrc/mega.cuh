@@ -79,6 +79,7 @@ struct MegaArgs {
     float *x;
     __nv_bfloat16 *act_d, *act_o, *act_f;
     float *q, *part, *attn_part, *top_part, *ssq;
+    float *cta_top;          // [gridDim.x][T_pad][4]: each CTA's top-2 over its own exit-head tiles (v1, id1, v2, -)
     const double *inv_freq;
     float2 *rope;            // [T_pad][hd / 2] (cos, sin) of each row's position, filled in the first phase
     int n_splits, n_mg, mt, G;
@@ -1154,33 +1155,48 @@ __device__ __forceinline__ bool mega_epilogue_head(const MegaGemm *g, const Mega
     return true;
 }
 
+// warps 4..7, after the CTA's exit-head tiles: one top-2 record per row over this CTA's own tile records, so that
+// the final reduction reads gridDim.x records per row instead of four per 128 vocabulary entries
+__device__ void mega_head_cta_merge(const MegaArgs &m, MegaShared &sh, int warp, int lane) {
+    asm volatile("bar.sync 2, 128;" ::: "memory");   // the four epilogue warps' records are written
+    const SegList &L = sh.segs[4][0];
+    const int n_rec = L.n * 4;
+    for (int t = warp - kWarpEpi0; t < m.T_pad; t += 4) {
+        Top2 best = {-INFINITY, -INFINITY, 0x7fffffff};
+        for (int i = lane; i < n_rec; i += 32) {
+            const int rec = L.tile[i >> 2] * 4 + (i & 3);
+            const float4 o = *reinterpret_cast<const float4 *>(m.top_part + ((size_t)rec * m.T_pad + t) * 4);
+            best = top2_merge(best, Top2{o.x, o.z, __float_as_int(o.y)});
+        }
+        best = top2_warp(best);
+        if (lane == 0)
+            *reinterpret_cast<float4 *>(m.cta_top + ((size_t)blockIdx.x * m.T_pad + t) * 4) =
+                make_float4(best.v1, __int_as_float(best.i1), best.v2, 0.f);
+    }
+}
+
 // ---- a9 (second half) + a10 for sequence b, by the worker threads of one CTA ---------------------
 __device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b) {
     const StageArgs &a = m.a;
     const AcceptArgs &r = m.r;
     const int nr = sh.nr[b];
-    const int wt = threadIdx.x - kMegaLeader, lane = threadIdx.x & 31, w = (threadIdx.x >> 5) - 1;
-    const int n_rec = m.head->tiles * 4;
-    for (int j = 0; j < nr; ++j) {
+    const int lane = threadIdx.x & 31, w = (threadIdx.x >> 5) - 1;
+    // one warp per row: the CTAs' records (one per CTA and row, written before the last grid barrier) in CTA order
+    for (int j = w; j < nr; j += kMegaWorkers / 32) {
         const int t = b * a.R_pad + j;
         Top2 best = {-INFINITY, -INFINITY, 0x7fffffff};
-        for (int rec = wt; rec < n_rec; rec += kMegaWorkers) {
-            const float *o = m.top_part + ((size_t)rec * m.T_pad + t) * 4;
-            best = top2_merge(best, Top2{o[0], o[2], __float_as_int(o[1])});
+        for (int c = lane; c < (int)gridDim.x; c += 32) {
+            const float4 o = *reinterpret_cast<const float4 *>(m.cta_top + ((size_t)c * m.T_pad + t) * 4);
+            best = top2_merge(best, Top2{o.x, o.z, __float_as_int(o.y)});
         }
         best = top2_warp(best);
-        worker_bar();
-        if (lane == 0) { sh.red_v1[w] = best.v1; sh.red_v2[w] = best.v2; sh.red_i1[w] = best.i1; }
-        worker_bar();
-        if (threadIdx.x == kMegaLeader) {
-            Top2 mm = {sh.red_v1[0], sh.red_v2[0], sh.red_i1[0]};
-            for (int i = 1; i < kMegaWorkers / 32; ++i) mm = top2_merge(mm, Top2{sh.red_v1[i], sh.red_v2[i], sh.red_i1[i]});
-            const float inv = mega_inv_rms(m, t);
-            m.argmax_ws[t] = mm.i1;
-            if (r.argmax_ids) r.argmax_ids[(size_t)b * a.max_rows + j] = mm.i1;
+        const float inv = mega_inv_rms_warp(m, t, lane);
+        if (lane == 0) {
+            m.argmax_ws[t] = best.i1;
+            if (r.argmax_ids) r.argmax_ids[(size_t)b * a.max_rows + j] = best.i1;
             if (r.top2) {
-                r.top2[((size_t)b * a.max_rows + j) * 2] = mm.v1 * inv;
-                r.top2[((size_t)b * a.max_rows + j) * 2 + 1] = mm.v2 * inv;
+                r.top2[((size_t)b * a.max_rows + j) * 2] = best.v1 * inv;
+                r.top2[((size_t)b * a.max_rows + j) * 2 + 1] = best.v2 * inv;
             }
         }
     }
@@ -1302,8 +1318,12 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
                 if (lane == 0) mega_x_load(kind, tmX[xbuf], ring, sh, xpos, m.status);
                 __syncwarp();
             } else {
-                if constexpr (decltype(head)::value) mega_epilogue_head(g, m, sh, seg_it, warp, lane);
-                else mega_epilogue_part(g, kind, m, sh, seg_it, warp, lane);
+                if constexpr (decltype(head)::value) {
+                    mega_epilogue_head(g, m, sh, seg_it, warp, lane);
+                    mega_head_cta_merge(m, sh, warp, lane);
+                } else {
+                    mega_epilogue_part(g, kind, m, sh, seg_it, warp, lane);
+                }
             }
             MEGA_STAMP(50 + kind);
             grid_sync(m, sh, false);   // partial sums / top-2 records: read by plain loads
@@ -1344,6 +1364,11 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         }
         gemm_phase(m.head, 4, 0, std::true_type{});
         for (int b = blockIdx.x; b < a.batch; b += gridDim.x) mega_accept(m, sh, b);
+        if (m.trace && blockIdx.x == 0 && threadIdx.x == kMegaLeader) {   // end of CTA 0's work (it finishes sequence 0)
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+            m.trace[1022] = t;
+        }
     }
     __syncthreads();
     if (warp == 2) {
