@@ -422,11 +422,13 @@ __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, c
         float v[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[i] = 0.f;
-        float4 p = make_float4(0.f, 0.f, 0.f, 0.f), q = p;
+        float4 p = make_float4(0.f, 0.f, 0.f, 0.f), q = p, g0 = p, g1 = p;
         if (c < m.d) {
             const float *xr = m.x + (size_t)t * m.d + c;
             p = *reinterpret_cast<const float4 *>(xr);
             q = *reinterpret_cast<const float4 *>(xr + 4);
+            g0 = *reinterpret_cast<const float4 *>(gain + c);   // fetched with everything else: the gain vector of a
+            g1 = *reinterpret_cast<const float4 *>(gain + c + 4);   // layer is cold, one more round trip if loaded at its use
             sum_slots8(m, g, t, c, v, hl, 2);
         }
 #pragma unroll
@@ -434,6 +436,7 @@ __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, c
             const float o = __shfl_xor_sync(0xffffffffu, v[i], 16);
             v[i] = hl ? o + v[i] : v[i] + o;   // first half + second half, the same value in both half-warps
         }
+        MEGA_STAMP(76);
         if (c < m.d) {
             const float xo[8] = {p.x, p.y, p.z, p.w, q.x, q.y, q.z, q.w};
 #pragma unroll
@@ -456,15 +459,17 @@ __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, c
                     *reinterpret_cast<float4 *>(e + 4) = make_float4(v[4], v[5], v[6], v[7]);
                 }
             } else {
+                const float gn[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
                 float gv[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) gv[i] = v[i] * gain[c + i];
+                for (int i = 0; i < 8; ++i) gv[i] = v[i] * gn[i];
                 store8_hilo(m.act_d + (size_t)t * m.d + c, m.act_d + ((size_t)m.T_alloc + t) * m.d + c, gv, m.plain);
             }
         }
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if (lane == 0) m.ssq[(size_t)t * nch + ch] = ss;
+        MEGA_STAMP(77);
     }
 }
 
@@ -499,10 +504,9 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         const float ssq = mega_ssq_fetch(m, t, lane);
         const int pos = sh.p0[b] + j;
         const int lp = pos / a.page_size, slot = pos % a.page_size;
+        // only loaded here: the check of the page id (a branch with a side effect) comes after the slot loads, which
+        // must not wait for this load's round trip
         const long long page = m.block_table[(size_t)b * a.max_pages + lp];
-        const bool page_ok = page >= 0 && page < m.n_pages;
-        if (!page_ok && lane == 0 && h == m.hq) atomicOr(m.status, HISPEC_ST_BOUNDS);
-        const size_t page_base = (((size_t)pool_layer * m.n_pages + (page_ok ? page : 0)) * m.hkv) * a.page_size * hd;
         // a head's columns lie in one 128-row weight tile (head_dim 64 or 128): one slot range for the item
         int first, ns;
         mega_slots((h * hd) / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
@@ -534,7 +538,12 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
                     for (int e = 0; e < 4; ++e) x[e] += u[e][k];   // slot order
                 }
         }
+        MEGA_STAMP(78);
         const float inv = mega_inv_rms_finish(m, ssq);
+        MEGA_STAMP(79);
+        const bool page_ok = page >= 0 && page < m.n_pages;
+        if (!page_ok && lane == 0 && h == m.hq) atomicOr(m.status, HISPEC_ST_BOUNDS);
+        const size_t page_base = (((size_t)pool_layer * m.n_pages + (page_ok ? page : 0)) * m.hkv) * a.page_size * hd;
         if (rot) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
