@@ -38,8 +38,11 @@ METRIC = "verified tokens/s per B200 (HiSpec, Llama-3-8B shape, batch 1, k=5)"
 UNIT = "tokens/s"
 N_PROMPT, N_D, ROUNDS = 1024, 5, 2
 # dram__bytes_read.sum + dram__bytes_write.sum of one hispec_stage_kernel launch (a verify-I call of this
-# workload: layers [8,16) + head, 6 rows, context 1024) from the ncu capture summarised under profiles/
-ROOFLINE_TRAFFIC_BYTES_PER_LAUNCH = 4.627e9
+# workload: layers [8,16) + head, 6 rows, context 1024, 4.576 GB algorithmic) from the ncu capture summarised
+# under profiles/.  The launches of a super-round differ in size (a block of 6 draft steps, a verify-I, a
+# verify-T); their traffic is that ratio times their algorithmic bytes (traffic is the weight stream, read once).
+ROOFLINE_TRAFFIC_BYTES_CAPTURED = 4.627e9
+ROOFLINE_TRAFFIC_RATIO = ROOFLINE_TRAFFIC_BYTES_CAPTURED / 4.576e9
 
 
 def peaks():
@@ -193,7 +196,7 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": "configs[1]: Llama-3-8B-shaped early-exit model, exits 8/16/32, batch 1, prompt 1024 "
                                "uniform-random tokens, k=5 greedy drafts, target every 2 intermediate rounds; "
                                "bf16 N(0,0.02) weights (literal: near-zero acceptance)",
-                   "step": "one super-round: 2 x (6 draft steps + verify-I) + verify-T", "replicas": world,
+                   "step": "one super-round: 2 x (6 draft steps as one call + verify-I) + verify-T", "replicas": world,
                    "l2": "inputs larger than L2 (each call streams >= 4.5 GB of weights)",
                    "activations": "bf16 hi+lo split", "tokens_committed": toks,
                    "algorithmic_gb_per_step": step_bytes / 1e9,
@@ -205,8 +208,10 @@ def run_ours(args, rank, world, local_rank):
                 "prompt_h2d_bytes": 4 * N_PROMPT},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": ROOFLINE_TRAFFIC_BYTES_PER_LAUNCH,
-                     "kernel": "hispec_stage_kernel (one launch = one whole draft / verify-I / verify-T call)",
+                     "traffic": ROOFLINE_TRAFFIC_RATIO * roof_bytes / max(g_n, 1),
+                     "traffic_note": "ncu DRAM read+write of a verify-I launch (4.627 GB for 4.576 GB algorithmic), "
+                                     "scaled to the average launch by algorithmic bytes",
+                     "kernel": "hispec_stage_kernel (one launch = one block of draft steps, one verify-I or one verify-T call)",
                      "launches": g_n, "avg_launch_us": 1e3 * g_ms / max(g_n, 1),
                      "algorithmic_bytes_per_launch": roof_bytes / max(g_n, 1), "weight_bytes_per_launch": g_wbytes / max(g_n, 1),
                      "peak_source": f"of {peak_kind}", "frac_of_8TBs": achieved / 8000.0},

@@ -156,6 +156,22 @@ int hispec_draft(hispec_ctx *ctx, void *stream, int layer_begin, int layer_end, 
                  int in_stride, int32_t *out_tokens, int out_stride, const hispec_result *res);
 
 /*
+ * Generate(L_d, ., N_d) (Algorithm 2) as ONE call: n_steps successive hispec_draft steps, plus one more if
+ * `bonus` is non-zero (its token is dropped: the step only pushes S_{N_d} through the draft layers so that the
+ * verifier can emit v_{N_d+1}).  Step 0 reads in_tokens[b * in_stride]; step s > 0 reads block[b * block_stride +
+ * s - 1]; step s < n_steps writes its greedy token to block[b * block_stride + s] (device int32, block_stride >=
+ * n_steps).  State, hidden rows and lengths change exactly as by the separate calls.  Where the persistent kernel
+ * takes the call, all steps run inside one launch (the weight stream continues from one step's exit head into
+ * the next step's first projection); otherwise the library issues the separate calls itself.  `res`, if given,
+ * holds the optional outputs of the last step.  The paper states Generate (Algorithm 2); fusing its steps into one
+ * launch is this library's.
+ */
+int hispec_draft_block(hispec_ctx *ctx, void *stream, int layer_begin, int layer_end, const hispec_exits *exits,
+                       const hispec_kv *kv, const hispec_hidden *hidden, int batch, const int32_t *in_tokens,
+                       int in_stride, int32_t *block, int block_stride, int n_steps, int bonus,
+                       const hispec_result *res);
+
+/*
  * LeadingSubstringVerify(S, L_i, x || V) (Algorithm 2): the n_rows[b] buffered exit-L_d rows of each
  * sequence run through layers [layer_begin, layer_end) (layer_begin == L_d; layer_end == L_i, or L_f
  * for single-stage speculation as in Algorithm 1) with causal attention inside the block and over

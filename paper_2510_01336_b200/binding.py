@@ -28,7 +28,7 @@ ST_BOUNDS, ST_STATE, ST_TIMEOUT = 1, 2, 4
 EXPORTS = ["hispec_create", "hispec_destroy", "hispec_draft", "hispec_verify_intermediate", "hispec_verify_target",
            "hispec_prefill", "hispec_device_status", "hispec_launch_count", "hispec_strerror",
            "hispec_profile_enable", "hispec_profile_read", "hispec_last_error", "hispec_exit_argmax_noalloc",
-           "hispec_debug_trace", "hispec_accept_rejection", "hispec_sample"]
+           "hispec_debug_trace", "hispec_accept_rejection", "hispec_sample", "hispec_draft_block"]
 
 
 class ModelDesc(ctypes.Structure):
@@ -100,6 +100,9 @@ def load() -> ctypes.CDLL:
         lib.hispec_accept_rejection.restype = ctypes.c_int
         lib.hispec_sample.argtypes = [vp, vp, i32, vp, ctypes.c_int64, vp, ctypes.c_float, vp, i32]
         lib.hispec_sample.restype = ctypes.c_int
+        lib.hispec_draft_block.argtypes = [vp, vp, i32, i32, ctypes.POINTER(CExits), ctypes.POINTER(CKv), ctypes.POINTER(CHidden),
+                                           i32, vp, i32, vp, i32, i32, i32, ctypes.POINTER(CResult)]
+        lib.hispec_draft_block.restype = ctypes.c_int
         for name in EXPORTS[:7] + EXPORTS[9:11]:
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
@@ -254,6 +257,17 @@ class Context:
         _check(self.lib.hispec_draft(self.handle, self._stream(stream), 0, le, ctypes.byref(self.exits),
                                      ctypes.byref(st.c_kv()), ctypes.byref(st.c_hidden()), b, ip, in_stride, op,
                                      out_stride, ctypes.byref(cres) if cres else None), "hispec_draft")
+
+    def draft_block(self, st: KVState, in_tokens, block: torch.Tensor, n_steps: int, bonus: bool = True,
+                    res: Optional[Result] = None, layer_end: Optional[int] = None, stream=None, in_stride: int = 1):
+        """Generate(L_d, ., n_steps) as one call: block [batch][stride >= n_steps] int32 receives the draft tokens."""
+        le = self.exits.L_d if layer_end is None else layer_end
+        cres = res.c() if res is not None else None
+        batch, stride = block.shape
+        _check(self.lib.hispec_draft_block(self.handle, self._stream(stream), 0, le, ctypes.byref(self.exits),
+                                           ctypes.byref(st.c_kv()), ctypes.byref(st.c_hidden()), batch, _ptr(in_tokens),
+                                           in_stride, _ptr(block), stride, n_steps, 1 if bonus else 0,
+                                           ctypes.byref(cres) if cres else None), "hispec_draft_block")
 
     def _verify(self, fn, name, st, l0, l1, draft_tokens, n_draft, n_rows, res, stream, k=None):
         batch, stride = draft_tokens.shape

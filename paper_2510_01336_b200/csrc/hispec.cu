@@ -561,6 +561,9 @@ struct StageCall {
     int token_stride, out_stride;
     const hispec_result *res;
     int32_t *out_tokens;
+    // a block of draft steps in one launch (0 steps: a plain call)
+    int32_t *block;
+    int block_stride, n_steps, bonus;
 };
 
 // one projection: activation buffer `which` (0: act_d, 1: act_o, 2: act_f) times weight matrix
@@ -731,6 +734,8 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         m.logits = sc.res->logits;
     }
     m.r.out_tokens = sc.out_tokens; m.r.n_tokens = sc.n_tokens;
+    m.n_rep = sc.block ? sc.n_steps + (sc.bonus ? 1 : 0) : 1;
+    m.block = sc.block; m.block_stride = sc.block_stride; m.n_steps = sc.n_steps;
     m.argmax_ws = c->argmax_ws;
     m.status = c->status;
     m.bar_count = x->bar + (x->bar_sel & 1); m.bar_next = x->bar + ((x->bar_sel + 1) & 1);
@@ -756,6 +761,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     c->launches++;
     double wbytes = 2.0 * (double)c->plan[G_HEAD].N * c->plan[G_HEAD].K;
     for (int k = 0; k < G_HEAD; ++k) wbytes += 2.0 * (double)c->plan[k].N * c->plan[k].K * (a.l1 - a.l0);
+    wbytes *= m.n_rep;
     ProfScope prof(c, st, 20, wbytes);
     cudaError_t le = (d.head_dim == 64)
                          ? cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m)
@@ -953,6 +959,34 @@ extern "C" int hispec_draft(hispec_ctx *c, void *stream, int l0, int l1, const h
     sc.exits = ex; sc.kv = kv; sc.hidden = hid; sc.tokens = in_tokens; sc.res = res; sc.out_tokens = out_tokens;
     sc.out_stride = out_stride;
     return run_stage(c, (cudaStream_t)stream, sc);
+}
+
+extern "C" int hispec_draft_block(hispec_ctx *c, void *stream, int l0, int l1, const hispec_exits *ex, const hispec_kv *kv,
+                                  const hispec_hidden *hid, int batch, const int32_t *in_tokens, int in_stride,
+                                  int32_t *block, int block_stride, int n_steps, int bonus, const hispec_result *res) {
+    int rc = check_common(c, l0, l1, ex, kv, batch);
+    if (rc) return rc;
+    if (l0 != 0 || !in_tokens || in_stride < 1 || !block || n_steps < 1 || block_stride < n_steps) return HISPEC_EINVAL;
+    if (l1 != ex->L_f && (!hid || !hid->h_draft || !hid->h_inter)) return HISPEC_EINVAL;
+    if (l1 != ex->L_f && n_steps + (bonus ? 1 : 0) > c->d.max_rows_per_seq) return HISPEC_EINVAL;
+    StageCall sc;
+    memset(&sc, 0, sizeof(sc));
+    sc.a = base_args(c, ex, l0, l1, batch, 1);
+    sc.a.mode = 0; sc.a.tok_stride = in_stride; sc.a.tok_offset = 0; sc.a.fixed_rows = 1;
+    sc.exits = ex; sc.kv = kv; sc.hidden = hid; sc.tokens = in_tokens; sc.res = res;
+    sc.block = block; sc.block_stride = block_stride; sc.n_steps = n_steps; sc.bonus = bonus ? 1 : 0;
+    if (!(c->d.flags & HISPEC_FLAG_MULTI_KERNEL)) {
+        rc = run_stage_mega(c, (cudaStream_t)stream, sc);
+        if (rc != 1) return rc;
+    }
+    // the persistent kernel does not take this call: the same steps as separate calls
+    const int total = n_steps + (bonus ? 1 : 0);
+    for (int s = 0; s < total; ++s) {
+        rc = hispec_draft(c, stream, l0, l1, ex, kv, hid, batch, s == 0 ? in_tokens : block + (s - 1),
+                          s == 0 ? in_stride : block_stride, s < n_steps ? block + s : nullptr, block_stride, res);
+        if (rc) return rc;
+    }
+    return HISPEC_OK;
 }
 
 extern "C" int hispec_verify_intermediate(hispec_ctx *c, void *stream, int l0, int l1, const hispec_exits *ex,

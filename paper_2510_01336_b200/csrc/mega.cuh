@@ -79,6 +79,10 @@ struct MegaArgs {
     float *x;
     __nv_bfloat16 *act_d, *act_o, *act_f;
     float *q, *part, *attn_part, *top_part, *ssq;
+    // a block of draft steps in one launch (hispec_draft_block): the call's steps a0..a10 run n_rep times; step s > 0
+    // reads its token from block[b * block_stride + s - 1], step s < n_steps writes block[b * block_stride + s]
+    int n_rep, n_steps, block_stride;
+    int32_t *block;
     float *cta_top;          // [gridDim.x][T_pad][4]: each CTA's top-2 over its own exit-head tiles (v1, id1, v2, -)
     const double *inv_freq;
     float2 *rope;            // [T_pad][hd / 2] (cos, sin) of each row's position, filled in the first phase
@@ -118,6 +122,12 @@ struct MegaShared {
     float red_v1[8], red_v2[8];
     int red_i1[8];
 };
+
+// token input / output of embedding-mode step `step` (a plain call has one step and block == nullptr)
+__device__ __forceinline__ int mega_tok_in(const MegaArgs &m, int step, int b, int j) {
+    if (step == 0 || !m.block) return m.tokens[b * m.a.tok_stride + m.a.tok_offset + j];
+    return m.block[(size_t)b * m.block_stride + step - 1];
+}
 
 // Development aid (compiled with -DHISPEC_STAMPS only): lane 0 of any warp of one CTA records
 // (tag * 100 + warp, global timer) pairs into the trace buffer, words 200.., while sh.stamp_on is set.
@@ -233,9 +243,9 @@ __device__ __forceinline__ void grid_sync(const MegaArgs &m, MegaShared &sh, boo
 }
 
 // ---- row bookkeeping (every CTA computes the same table; CTA 0 reports) -------------------------
-__device__ __forceinline__ void mega_prep_rows(const MegaArgs &m, MegaShared &sh) {
+__device__ __forceinline__ void mega_prep_rows(const MegaArgs &m, MegaShared &sh, int step, int tid, int nthreads) {
     const StageArgs &a = m.a;
-    for (int b = threadIdx.x; b < a.batch; b += blockDim.x) {
+    for (int b = tid; b < a.batch; b += nthreads) {
         int gA = m.len_d[b], gB = m.len_i[b], gC = m.len_f[b];
         int p0 = a.l0 < a.L_d ? gA : (a.l0 < a.L_i ? gB : gC);
         uint32_t st = 0;
@@ -246,7 +256,7 @@ __device__ __forceinline__ void mega_prep_rows(const MegaArgs &m, MegaShared &sh
                 nr = nr < 0 ? 0 : (nr > a.R_pad ? a.R_pad : nr);
             } else {
                 nr = a.fixed_rows;
-                if (m.tokens[b * a.tok_stride + a.tok_offset] < 0) nr = 0;
+                if (mega_tok_in(m, step, b, 0) < 0) nr = 0;
             }
         } else if (m.n_rows_in) {
             nr = m.n_rows_in[b];
@@ -344,7 +354,7 @@ __device__ __forceinline__ float sum_slots1(const MegaArgs &m, const MegaGemm &g
 
 // ---- element-wise phases (gw: global worker-warp index, ngw: number of worker warps in the grid) ----
 // a0 + gain: fetch rows, x <- row, act_d <- hi/lo(x .* gain), chunk sums of squares
-__device__ void ew_rows_in(const MegaArgs &m, MegaShared &sh, const float *gain, int gw, int ngw, int lane) {
+__device__ void ew_rows_in(const MegaArgs &m, MegaShared &sh, const float *gain, int step, int gw, int ngw, int lane) {
     const StageArgs &a = m.a;
     const int nch = (m.d + kEwChunk - 1) / kEwChunk;
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
@@ -356,7 +366,7 @@ __device__ void ew_rows_in(const MegaArgs &m, MegaShared &sh, const float *gain,
         for (int i = 0; i < 8; ++i) v[i] = 0.f;
         if (valid && c < m.d) {
             if (a.mode == 0) {
-                int tok = m.tokens[b * a.tok_stride + a.tok_offset + j];
+                int tok = mega_tok_in(m, step, b, j);
                 if (tok < 0 || tok >= m.vocab) {
                     if (lane == 0 && ch == 0) atomicOr(m.status, HISPEC_ST_BOUNDS);
                 } else {
@@ -884,6 +894,7 @@ struct WCursor {
     const MegaShared *sh;
     int p;
     int gi, n_g;   // projection index in call order; 4 per layer, then the exit head
+    int rep;       // step of a block of draft steps (the same projections again)
     int si, tile, kb, kb1;
     bool valid;
     __device__ int kind() const { return gi + 1 < n_g ? (gi & 3) : 4; }
@@ -891,7 +902,7 @@ struct WCursor {
         return gi + 1 < n_g ? &m->gemms[(m->a.l0 + (gi >> 2)) * 4 + (gi & 3)] : m->head;
     }
     __device__ WCursor(const MegaArgs *m_, const MegaShared *sh_, int p_)
-        : m(m_), sh(sh_), p(p_), gi(0), n_g(4 * (m_->a.l1 - m_->a.l0) + 1), si(-1), tile(0), kb(0), kb1(0), valid(true) {
+        : m(m_), sh(sh_), p(p_), gi(0), n_g(4 * (m_->a.l1 - m_->a.l0) + 1), rep(0), si(-1), tile(0), kb(0), kb1(0), valid(true) {
         advance();
     }
     __device__ void advance() {
@@ -900,7 +911,10 @@ struct WCursor {
             const SegList &L = sh->segs[kind()][p];
             if (++si < L.n) { tile = L.tile[si]; kb = L.kb0[si]; kb1 = L.kb1[si]; return; }
             si = -1;
-            if (++gi >= n_g) { valid = false; return; }
+            if (++gi >= n_g) {
+                if (++rep >= m->n_rep) { valid = false; return; }
+                gi = 0;
+            }
         }
     }
 };
@@ -948,7 +962,7 @@ __device__ __forceinline__ bool mega_w_issue(const MegaArgs &m, int p, WLane &w,
     w.last_ph = w.pos.ph;
     w.ld.advance();
     w.pos.advance(ring.stages);
-    if (w.ld.valid && w.ld.gi != w.cur_gi) { w.cur_gi = w.ld.gi; w.gate = true; }
+    if (w.ld.valid && w.ld.gi + w.ld.rep * w.ld.n_g != w.cur_gi) { w.cur_gi = w.ld.gi + w.ld.rep * w.ld.n_g; w.gate = true; }
     return true;
 }
 __device__ __forceinline__ void mega_w_producer(const MegaArgs &m, const MegaRing *ring, MegaShared &sh) {
@@ -1185,7 +1199,7 @@ __device__ void mega_head_cta_merge(const MegaArgs &m, MegaShared &sh, int warp,
 }
 
 // ---- a9 (second half) + a10 for sequence b, by the worker threads of one CTA ---------------------
-__device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b) {
+__device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b, int step) {
     const StageArgs &a = m.a;
     const AcceptArgs &r = m.r;
     const int nr = sh.nr[b];
@@ -1239,7 +1253,9 @@ __device__ void mega_accept(const MegaArgs &m, MegaShared &sh, int b) {
         m.len_d[b] = nl;
         if (a.l1 > a.L_d) m.len_i[b] = nl;
         if (a.l1 > a.L_i) m.len_f[b] = nl;
-        if (r.out_tokens) {
+        if (m.block) {   // a block of draft steps: the token feeds the next step; the bonus step's token is dropped
+            if (step < m.n_steps) m.block[(size_t)b * m.block_stride + step] = m.argmax_ws[b * a.R_pad + nr - 1];
+        } else if (r.out_tokens) {
             bool emit = true;
             if (r.n_tokens) emit = (nl == r.n_tokens[b]);
             if (emit) r.out_tokens[(size_t)b * r.out_stride] = m.argmax_ws[b * a.R_pad + nr - 1];
@@ -1302,7 +1318,7 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    mega_prep_rows(m, sh);
+    mega_prep_rows(m, sh, 0, threadIdx.x, blockDim.x);
     mega_fill_seglists(m, sh);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -1337,7 +1353,13 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
             MEGA_STAMP(50 + kind);
             grid_sync(m, sh, false);   // partial sums / top-2 records: read by plain loads
         };
-        ew_rows_in(m, sh, m.attn_norm[a.l0], gw, ngw, lane);
+        for (int step = 0; step < m.n_rep; ++step) {
+        if (step > 0) {   // a block of draft steps: the previous step's tokens and lengths are final after this barrier
+            grid_sync(m, sh, false);
+            mega_prep_rows(m, sh, step, threadIdx.x - kMegaLeader, kMegaWorkers);
+            worker_bar();
+        }
+        ew_rows_in(m, sh, m.attn_norm[a.l0], step, gw, ngw, lane);
         ew_rope_table(m, sh, gw, ngw, lane);
         grid_sync(m, sh);
         for (int l = a.l0; l < a.l1; ++l) {
@@ -1372,7 +1394,8 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
             }
         }
         gemm_phase(m.head, 4, 0, std::true_type{});
-        for (int b = blockIdx.x; b < a.batch; b += gridDim.x) mega_accept(m, sh, b);
+        for (int b = blockIdx.x; b < a.batch; b += gridDim.x) mega_accept(m, sh, b, step);
+        }
         if (m.trace && blockIdx.x == 0 && threadIdx.x == kMegaLeader) {   // end of CTA 0's work (it finishes sequence 0)
             unsigned long long t;
             asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));

@@ -38,10 +38,11 @@ class HiSpecLoop:
     acceptance outcome is per sequence)."""
 
     def __init__(self, ctx: binding.Context, st: binding.KVState, batch: int, N_d: int, rounds: int = 2,
-                 bonus_inter: bool = True, device: str = "cuda"):
+                 bonus_inter: bool = True, device: str = "cuda", block_drafts: bool = True):
         per_round = N_d + (1 if bonus_inter else 0)
         assert per_round * rounds <= ctx.max_rows - 1, "hidden buffers too small: need rounds * (N_d + 1) + 1 rows"
         self.ctx, self.st, self.B, self.N_d, self.rounds, self.bonus = ctx, st, batch, N_d, rounds, bonus_inter
+        self.block_drafts = block_drafts   # Generate(L_d, ., N_d) as one library call instead of N_d (+1)
         i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device=device)
         self.pending = i32(batch)                      # token waiting to enter the draft layers
         self.S = i32(batch, N_d)                       # draft block of the current round
@@ -83,15 +84,19 @@ class HiSpecLoop:
         S_ptr = self.S.data_ptr()
         for r in range(self.rounds):
             src = self.pending  # kept current by the acceptance kernel of the previous verification
-            # Generate(L_d, ., N_d): step j reads column j-1 of S (or the pending token) and writes column j
-            for j in range(N_d):
-                if j == 0:
-                    ctx.draft(st, src, S_ptr, batch=B, in_stride=1, out_stride=N_d, stream=stream)
-                else:
-                    ctx.draft(st, S_ptr + 4 * (j - 1), S_ptr + 4 * j, batch=B, in_stride=N_d, out_stride=N_d,
-                              stream=stream)
-            if self.bonus:  # push S_{N_d} through the draft layers so that L_i can emit v_{N_d+1}
-                ctx.draft(st, S_ptr + 4 * (N_d - 1), None, batch=B, in_stride=N_d, stream=stream)
+            if self.block_drafts:
+                # Generate(L_d, ., N_d) as one call: all draft steps (and the bonus step) inside one launch
+                ctx.draft_block(st, src, self.S, N_d, bonus=self.bonus, stream=stream)
+            else:
+                # step j reads column j-1 of S (or the pending token) and writes column j
+                for j in range(N_d):
+                    if j == 0:
+                        ctx.draft(st, src, S_ptr, batch=B, in_stride=1, out_stride=N_d, stream=stream)
+                    else:
+                        ctx.draft(st, S_ptr + 4 * (j - 1), S_ptr + 4 * j, batch=B, in_stride=N_d, out_stride=N_d,
+                                  stream=stream)
+                if self.bonus:  # push S_{N_d} through the draft layers so that L_i can emit v_{N_d+1}
+                    ctx.draft(st, S_ptr + 4 * (N_d - 1), None, batch=B, in_stride=N_d, stream=stream)
             ctx.verify_intermediate(st, self.S, None, None, self.res_i[r], stream=stream, k=N_d)
             self.stats.draft_steps += N_d + (1 if self.bonus else 0)
             self.stats.inter_calls += 1

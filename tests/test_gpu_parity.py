@@ -205,6 +205,51 @@ def test_tiny_dynamic_trigger_and_single_stage_loops_are_lossless():
     assert outs["dynamic"] == outs["ar"] and outs["selfspec"] == outs["ar"]
 
 
+@pytest.mark.parametrize("flagname", ["tcgen05", "multi-kernel"])
+def test_draft_block_equals_separate_draft_steps(flagname):
+    """hispec_draft_block (all draft steps of a round in one call) against the same steps as separate calls:
+    the same tokens, length counters, buffered exit rows and appended K/V, bit for bit."""
+    b = _binding()
+    shape = wl.TINY
+    wg = wl.make_weights(shape).to("cuda")
+    flags = {"tcgen05": 0, "multi-kernel": b.FLAG_MULTI_KERNEL}[flagname]
+    B, N_d, n_prompt = 3, 4, 40
+    max_rows, max_pages = 8, 6
+    prompts = [wl.make_tokens(shape, n_prompt - 3 * s, seed_offset=1000 + s).tolist() for s in range(B)]
+    bt = wl.make_block_table(shape, B, max_pages)
+    outs = []
+    for mode in ("separate", "block"):
+        ctx = b.Context(shape, wg, max_batch=B, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages, flags=flags)
+        st = ctx.new_state(B, B * max_pages, bt)
+        mx = max(len(p) for p in prompts)
+        toks = torch.zeros((B, mx), dtype=torch.int32)
+        for s_, p in enumerate(prompts):
+            toks[s_, : len(p)] = torch.tensor(p, dtype=torch.int32)
+        pending = torch.zeros(B, dtype=torch.int32, device="cuda")
+        ctx.prefill(st, toks.cuda(), torch.tensor([len(p) for p in prompts], dtype=torch.int32).cuda(), pending)
+        S = torch.full((B, N_d), -1, dtype=torch.int32, device="cuda")
+        for rnd in range(2):      # two rounds in a row: the second starts from the first one's state
+            if mode == "block":
+                ctx.draft_block(st, pending, S, N_d, bonus=True)
+            else:
+                p_ = S.data_ptr()
+                ctx.draft(st, pending, p_, batch=B, in_stride=1, out_stride=N_d)
+                for j in range(1, N_d):
+                    ctx.draft(st, p_ + 4 * (j - 1), p_ + 4 * j, batch=B, in_stride=N_d, out_stride=N_d)
+                ctx.draft(st, p_ + 4 * (N_d - 1), None, batch=B, in_stride=N_d)
+            if rnd == 0:          # accept nothing: prune the draft group back by hand to one token past the start
+                S0 = S.clone()
+                st.len_draft.copy_(st.len_inter + 1)
+                pending = S0[:, 0].contiguous()
+        assert ctx.status() == 0
+        outs.append((S0.cpu(), S.cpu(), st.len_draft.cpu(), st.len_inter.cpu(), st.h_draft.cpu().clone(),
+                     st.k_pages.cpu().clone(), st.v_pages.cpu().clone()))
+        ctx.close()
+    for x, y in zip(*outs):
+        assert torch.equal(x, y)
+    assert int(outs[0][2][0]) == len(prompts[0]) + 1 + N_d + 1
+
+
 def test_tiny_adaptive_parameters_loop_is_lossless():
     """Adaptive N_d / N_i (App. J) free-running on the GPU: the output equals the GPU's own auto-regressive
     greedy output, both parameters move, and the recorded schedule obeys the oracle's update rule."""
