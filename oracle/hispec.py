@@ -579,6 +579,72 @@ class HiSpecOracle:
         stats.committed = min(len(x) - n0, n_gen)
         return x[n0: n0 + n_gen]
 
+    # ------------------------------------------------ several intermediate verifiers (App. K, future work)
+    def chain_generate(self, prompt: Sequence[int], n_gen: int, exits: Sequence[int], N_d: int,
+                       rounds: Sequence[int], schedule: Optional[list] = None) -> List[int]:
+        """HiSpec with a chain of verifiers L_d = exits[0] < exits[1] < ... < exits[K] = L_f (App. K): level 1
+        filters the draft blocks as in Algorithm 2; level l > 1 runs LeadingSubstringVerify on the list that
+        level l - 1 has accumulated over rounds[l - 2] of its rounds; the last level is the target.  Every level
+        keeps the exit rows of the level below (Sec. 3.2 applied per level) and every verification prunes all
+        shallower layer groups.  len(rounds) == K - 1.  Written on the model primitives, with its own state, so
+        that it does not lean on the three-exit stage calls; the output must equal greedy decoding from L_f."""
+        K = len(exits) - 1
+        assert K >= 1 and len(rounds) == K - 1 and list(exits) == sorted(set(exits)) and exits[-1] <= self.m.n_layers
+        cap_rows = (N_d + 1) * int(np.prod([max(1, r) for r in rounds]) if rounds else 1) + 2
+        cache = self.m.new_cache(len(prompt) + n_gen + 2 * cap_rows + 4)
+        d = self.m.d_model
+        H = [np.zeros((cap_rows, d), np.float32) for _ in range(K)]     # H[g]: exit rows of level g, relative to lens[g + 1]
+        x0 = np.stack([self.m.embed(t) for t in prompt])
+        self.m.forward(0, exits[-1], x0, 0, cache)
+        lens = [len(prompt)] * (K + 1)                                   # lens[g]: valid KV length of layers [exits[g-1], exits[g])
+        pending = self._exit(x0[-1:]).argmax_ids[0]
+        x = [int(t) for t in prompt] + [pending]
+        n0 = len(prompt)
+
+        def verify(level: int, block: List[int], R: int) -> List[int]:
+            p0 = lens[level]
+            rows = H[level - 1][:R].copy()
+            self.m.forward(exits[level - 1], exits[level], rows, p0, cache)
+            if level < K:
+                base = lens[level] - lens[level + 1]
+                H[level][base: base + R] = rows
+            ids = self._exit(rows).argmax_ids
+            res, a = leading_substring_verify(block, ids[:R])
+            for g in range(level + 1):
+                lens[g] = p0 + min(a + 1, R)
+            if schedule is not None:
+                schedule.append((level, len(block), a))
+            return res
+
+        def produce(level: int) -> List[int]:
+            """The list tentatively accepted at `level` after rounds[level - 1] of its rounds (level K: one round)."""
+            nonlocal pending
+            out: List[int] = []
+            for _ in range(rounds[level - 1] if level < K else 1):
+                if level == 1:
+                    S, u = [], pending
+                    for j in range(N_d + 1):                 # N_d drafts and the bonus step
+                        row = self.m.embed(u)[None, :].copy()
+                        self.m.forward(0, exits[0], row, lens[0], cache)
+                        H[0][lens[0] - lens[1]] = row[0]
+                        lens[0] += 1
+                        if j < N_d:
+                            u = self._exit(row).argmax_ids[0]
+                            S.append(u)
+                    res = verify(1, S, N_d + 1)
+                else:
+                    block = produce(level - 1)
+                    res = verify(level, block, len(block))
+                out += res
+                pending = out[-1]
+            return out
+
+        while len(x) - n0 < n_gen:
+            F = produce(K)
+            x += F
+            pending = F[-1]
+        return x[n0: n0 + n_gen]
+
     def _generate_observed(self, st, pending, N_d, bonus, stats, draft_override, observer, ctx_tokens):
         S, u = [], pending
         for j in range(N_d + (1 if bonus else 0)):

@@ -161,3 +161,24 @@ def test_acceptance_bookkeeping_matches_closed_form(alpha):
     expect = alpha * (1 - alpha ** k) / (1 - alpha)
     se = 1.5 / np.sqrt(blocks)
     assert abs(mean - expect) < 4 * se, (mean, expect, blocks)
+
+
+def test_chain_of_verifiers_is_lossless():
+    """Several intermediate verifiers (App. K): whatever the chain, the output is greedy decoding from L_f; with
+    one verifier level the chain is Algorithm 1, with two it is Algorithm 2 with a fixed number of rounds."""
+    from paper_2510_01336_b200 import workload as wl
+    from tests.helpers import oracle_for
+    import dataclasses
+    shape = dataclasses.replace(wl.MINI_GQA, L_d=1, L_i=3, L_f=6)
+    scale = {l: 0.05 for l in range(1, 6)}
+    _, _, hs = oracle_for(shape, resid_scale=scale)
+    prompt = wl.make_tokens(shape, 12).tolist()
+    n_gen = 20
+    ar = hs.ar_generate(prompt, n_gen)
+    sched = []
+    assert hs.chain_generate(prompt, n_gen, [1, 2, 4, 6], 2, [2, 2], schedule=sched) == ar
+    assert {lv for lv, _, _ in sched} == {1, 2, 3}
+    assert sum(a for lv, _, a in sched if lv == 1) > 0 and sum(a for lv, _, a in sched if lv == 3) > 0
+    assert hs.chain_generate(prompt, n_gen, [1, 3, 6], 2, [2]) == hs.hispec_generate(prompt, n_gen, 2, rounds=2)
+    assert hs.chain_generate(prompt, n_gen, [1, 3, 6], 2, [2]) == ar
+    assert hs.chain_generate(prompt, n_gen, [2, 6], 3, []) == ar
