@@ -345,6 +345,119 @@ class HiSpecSamplingLoop(HiSpecLoop):
         self.stats.super_rounds += 1
 
 
+class HiSpecChainLoop:
+    """HiSpec with TWO intermediate verifiers, exits e0 < e1 < e2 < e3 (App. K, "multiple intermediate
+    verifiers"), through the three-exit ABI: the library is given two overlapping views of the same state --
+    view A = (e0, e1, e2) with the length counters (len0, len1, len2) and hidden buffers (h0, h1), view B =
+    (e1, e2, e3) with (len1, len2, len3) and (h1, h2).  Drafts and the first verifier are view A's draft and
+    intermediate-verification calls; the second verifier is view B's intermediate verification (rows from h1,
+    exit rows appended to h2, its result list appended to V2); the target is view B's target verification.  A
+    call of view B prunes len1..len3 but does not know layer group 0: a copy len1 -> len0 follows it.  One
+    super-round = m2 x [ m1 x (N_d drafts + bonus, verify at e1), verify at e2 ], verify at e3; no host
+    synchronisation inside."""
+
+    def __init__(self, shape, weights, exits, batch: int, N_d: int, m1: int, m2: int, max_pages: int, block_table,
+                 page_size: int = 16, device: str = "cuda"):
+        e0, e1, e2, e3 = exits
+        assert 0 < e0 < e1 < e2 < e3 <= shape.n_layers
+        rows1 = m1 * (N_d + 1)                 # rows level 1 can accumulate before level 2 runs
+        rows2 = m2 * rows1                     # ... level 2 before the target runs
+        self.max_rows = rows2 + 2
+        self.A = binding.Context(shape, weights, page_size=page_size, max_batch=batch, max_rows_per_seq=self.max_rows,
+                                 max_pages_per_seq=max_pages, exits=(e0, e1, e2))
+        self.Bc = binding.Context(shape, weights, page_size=page_size, max_batch=batch, max_rows_per_seq=self.max_rows,
+                                  max_pages_per_seq=max_pages, exits=(e1, e2, e3))
+        self.B, self.N_d, self.m1, self.m2 = batch, N_d, m1, m2
+        stA = self.A.new_state(batch, int(block_table.max()) + 1, block_table)
+        i32 = lambda *sh: torch.zeros(sh, dtype=torch.int32, device=device)
+        f32 = lambda *sh: torch.zeros(sh, dtype=torch.float32, device=device)
+        self.len = [stA.len_draft, stA.len_inter, stA.len_target, i32(batch)]      # len0..len3
+        self.h = [stA.h_draft, stA.h_inter, f32(batch, self.max_rows, shape.d_model)]
+        self.stA = stA
+        self.stB = binding.KVState(stA.k_pages, stA.v_pages, stA.block_table, self.len[1], self.len[2], self.len[3],
+                                   self.h[1], self.h[2], 0)
+        self.pending = i32(batch)
+        self.S = i32(batch, N_d)
+        self.V1 = i32(batch, self.max_rows)
+        self.V2 = i32(batch, self.max_rows)
+        mk = lambda tent: binding.Result(i32(batch), i32(batch), tentative=tent, pending=self.pending)
+        self.res1 = [mk(self.V1) for _ in range(m1 * m2)]
+        self.res2 = [mk(self.V2) for _ in range(m2)]
+        self.res3 = mk(None)
+        self.h_acc = torch.zeros(batch, dtype=torch.int32).pin_memory()
+        self.h_next = torch.zeros(batch, dtype=torch.int32).pin_memory()
+        self.h_V2 = torch.zeros((batch, self.max_rows), dtype=torch.int32).pin_memory()
+        self.tokens: List[List[int]] = [[] for _ in range(batch)]
+        self.stats = LoopStats()
+
+    def close(self):
+        self.A.close(); self.Bc.close()
+
+    def status(self) -> int:
+        return self.A.status() | self.Bc.status()
+
+    def prefill(self, prompts: List[List[int]]):
+        B = self.B
+        mx = max(len(p) for p in prompts)
+        toks = torch.zeros((B, mx), dtype=torch.int32)
+        for b, p in enumerate(prompts):
+            toks[b, : len(p)] = torch.tensor(p, dtype=torch.int32)
+        n = torch.tensor([len(p) for p in prompts], dtype=torch.int32).cuda()
+        # view B's prefill runs the prompt through all layers [0, e3) and sets its three counters; group 0 follows
+        self.Bc.prefill(self.stB, toks.cuda(), n, self.pending)
+        self.len[0].copy_(self.len[1])
+        torch.cuda.synchronize()
+        first = self.pending.cpu().tolist()
+        for b in range(B):
+            self.tokens[b] = [first[b]]
+        return first
+
+    def enqueue_super_round(self, stream=None):
+        A, Bc, N_d = self.A, self.Bc, self.N_d
+        s = stream if stream is not None else torch.cuda.current_stream()
+        r1 = 0
+        for i2 in range(self.m2):
+            for i1 in range(self.m1):
+                A.draft_block(self.stA, self.pending, self.S, N_d, bonus=True, stream=stream)
+                A.verify_intermediate(self.stA, self.S, None, None, self.res1[r1], stream=stream, k=N_d)
+                r1 += 1
+                self.stats.draft_steps += N_d + 1
+                self.stats.inter_calls += 1
+            # second verifier: LeadingSubstringVerify(V1, e2, .) on the rows level 1 has buffered
+            Bc.verify_intermediate(self.stB, self.V1, None, None, self.res2[i2], stream=stream, k=self.max_rows - 1)
+            with torch.cuda.stream(s):
+                self.len[0].copy_(self.len[1])
+            self.stats.inter_calls += 1
+        Bc.verify_target(self.stB, self.V2, None, None, self.res3, stream=stream, k=self.max_rows - 1)
+        with torch.cuda.stream(s):
+            self.len[0].copy_(self.len[1])
+        self.stats.target_calls += 1
+        self.stats.super_rounds += 1
+
+    def collect(self, stream=None):
+        s = stream if stream is not None else torch.cuda.current_stream()
+        with torch.cuda.stream(s):
+            self.h_acc.copy_(self.res3.n_accepted, non_blocking=True)
+            self.h_next.copy_(self.res3.next_token, non_blocking=True)
+            self.h_V2.copy_(self.V2, non_blocking=True)
+        s.synchronize()
+        new = []
+        for b in range(self.B):
+            a, nxt = int(self.h_acc[b]), int(self.h_next[b])
+            F = self.h_V2[b, :a].tolist() + ([nxt] if nxt >= 0 else [])
+            self.tokens[b] += F
+            new.append(F)
+            self.stats.target_accepted += a
+            self.stats.committed += len(F)
+        return new
+
+    def generate(self, n_gen: int) -> List[List[int]]:
+        while min(len(t) for t in self.tokens) < n_gen:
+            self.enqueue_super_round()
+            self.collect()
+        return [t[:n_gen] for t in self.tokens]
+
+
 class SelfSpecLoop:
     """Algorithm 1 (single-stage self-speculation): N_d (+1) draft steps at L_d, then one verification of the
     block by the final layer -- hispec_verify_intermediate over [L_d, L_f) with the L_f exit."""

@@ -250,6 +250,35 @@ def test_draft_block_equals_separate_draft_steps(flagname):
     assert int(outs[0][2][0]) == len(prompts[0]) + 1 + N_d + 1
 
 
+def test_tiny_chain_of_two_intermediate_verifiers_is_lossless():
+    """Two intermediate verifiers (exits 1 < 2 < 3 < 4, App. K) composed from the three-exit calls: the output
+    equals the GPU's own auto-regressive greedy output, and every level accepted something."""
+    b = _binding()
+    from paper_2510_01336_b200.driver import ARLoop, HiSpecChainLoop
+    shape = wl.TINY
+    scale = {l: 0.05 for l in range(1, shape.n_layers)}
+    wg = wl.make_weights(shape, resid_scale=scale).to("cuda")
+    B, n_prompt, n_gen, N_d, m1, m2 = 2, 48, 40, 2, 2, 2
+    max_pages = (n_prompt + n_gen + 40) // 16 + 1
+    prompts = [wl.make_tokens(shape, n_prompt - 5 * s, seed_offset=1000 + s).tolist() for s in range(B)]
+    bt = wl.make_block_table(shape, B, max_pages)
+    loop = HiSpecChainLoop(shape, wg, (1, 2, 3, 4), B, N_d, m1, m2, max_pages, bt)
+    loop.prefill(prompts)
+    toks = loop.generate(n_gen)
+    assert loop.status() == 0
+    acc1 = sum(int(r.n_accepted.sum()) for r in loop.res1)
+    acc2 = sum(int(r.n_accepted.sum()) for r in loop.res2)
+    assert acc1 > 0 and acc2 > 0 and loop.stats.target_accepted > 0
+    assert loop.stats.inter_calls == loop.stats.super_rounds * (m1 * m2 + m2)
+    loop.close()
+    ctx = b.Context(shape, wg, max_batch=B, max_rows_per_seq=4, max_pages_per_seq=max_pages)
+    st = ctx.new_state(B, int(bt.max()) + 1, bt)
+    ar = ARLoop(ctx, st, B)
+    ar.prefill(prompts)
+    assert toks == ar.generate(n_gen)
+    ctx.close()
+
+
 def test_tiny_adaptive_parameters_loop_is_lossless():
     """Adaptive N_d / N_i (App. J) free-running on the GPU: the output equals the GPU's own auto-regressive
     greedy output, both parameters move, and the recorded schedule obeys the oracle's update rule."""
