@@ -302,4 +302,163 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
 }
 
+
+// ---- the same projection for many rows (more than 64): two weight tiles per CTA share one activation tile ------
+// With T rows the activation tile of a k-block is T x 128 bytes per plane -- larger than the 16 KiB weight tile from
+// 64 rows on -- and it is re-read for every weight tile.  Here a CTA takes TWO adjacent weight tiles (256 output
+// features) per activation tile, which halves that traffic and leaves room for a deeper ring of weight blocks (one
+// CTA per SM, all of its shared memory).  Both planes of the activations accumulate into the SAME accumulator
+// (W.hi + W.lo is what the epilogue would add anyway), so an accumulator has t_box <= 256 columns: tile 0 at
+// column 0, tile 1 at column 256.
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[16], bar_empty[16], bar_acc;
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pair = blockIdx.x, sp = blockIdx.y;
+    const int tile0 = 2 * pair;
+    const bool two = (tile0 + 1) * kWeightTileRows < g.N;   // the second tile exists
+    const int kb0 = (int)((long long)g.kb_total * sp / g.splits);
+    const int kb1 = (int)((long long)g.kb_total * (sp + 1) / g.splits);
+    const int nkb = kb1 - kb0;
+    const uint32_t x_bytes = (uint32_t)(g.t_box * g.planes) * 128u;
+    const uint32_t w_bytes = two ? 2u * kWTileBytes : kWTileBytes;
+    const uint32_t stage_bytes = 2u * kWTileBytes + x_bytes;
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    volatile int *abort_flag = &s_abort;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < g.stages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_acc), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = s_tmem;
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint64_t policy = l2_policy_evict_first();
+            auto load_w = [&](int s, int kb) {
+                const uint32_t fb = smem_u32(&bar_full[s]);
+                mbar_expect_tx(fb, w_bytes + x_bytes);
+                tma_load_2d_stream(smem0 + s * stage_bytes, &tmW, kb * kTileK, tile0 * kWeightTileRows, fb, policy);
+                if (two)
+                    tma_load_2d_stream(smem0 + s * stage_bytes + kWTileBytes, &tmW, kb * kTileK, (tile0 + 1) * kWeightTileRows, fb,
+                                       policy);
+            };
+            // weights do not depend on the previous kernel: fill the ring with them first
+            const int pre = nkb < g.stages ? nkb : g.stages;
+            for (int i = 0; i < pre; ++i) load_w(i, kb0 + i);
+            pdl_wait();
+            for (int i = 0; i < pre; ++i)
+                tma_load_3d(smem0 + i * stage_bytes + 2 * kWTileBytes, &tmX, (kb0 + i) * kTileK, g.row0, 0, smem_u32(&bar_full[i]));
+            int s = pre == g.stages ? 0 : pre;
+            uint32_t ph = pre == g.stages ? 1u : 0u;
+            for (int i = pre; i < nkb; ++i) {
+                if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, abort_flag, g.status)) break;
+                load_w(s, kb0 + i);
+                tma_load_3d(smem0 + s * stage_bytes + 2 * kWTileBytes, &tmX, (kb0 + i) * kTileK, g.row0, 0, smem_u32(&bar_full[s]));
+                if (++s == g.stages) { s = 0; ph ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(g.t_box);
+            const uint64_t lo_off = (uint64_t)((g.t_box * 128) >> 4);   // the lo plane sits t_box rows further on
+            bool ok = true;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int i = 0; i < nkb && ok; ++i) {
+                ok = mbar_wait(smem_u32(&bar_full[s]), ph, abort_flag, g.status);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t a0 = umma_desc_sw128(smem0 + s * stage_bytes);
+                const uint64_t a1 = umma_desc_sw128(smem0 + s * stage_bytes + kWTileBytes);
+                const uint64_t bd = umma_desc_sw128(smem0 + s * stage_bytes + 2 * kWTileBytes);
+#pragma unroll
+                for (int k = 0; k < kTileK / 16; ++k) {
+                    const uint64_t kk = (uint64_t)(2 * k);
+                    umma_bf16(tmem_d, a0 + kk, bd + kk, idesc, (i | k) ? 1u : 0u);
+                    if (g.planes == 2) umma_bf16(tmem_d, a0 + kk, bd + lo_off + kk, idesc, 1u);
+                    if (two) {
+                        umma_bf16(tmem_d + 256u, a1 + kk, bd + kk, idesc, (i | k) ? 1u : 0u);
+                        if (g.planes == 2) umma_bf16(tmem_d + 256u, a1 + kk, bd + lo_off + kk, idesc, 1u);
+                    }
+                }
+                umma_commit(smem_u32(&bar_empty[s]));
+                if (++s == g.stages) { s = 0; ph ^= 1u; }
+            }
+            umma_commit(smem_u32(&bar_acc));
+        }
+    } else {
+        pdl_wait();
+        const int lg = warp & 3;
+        const bool ok = mbar_wait(smem_u32(&bar_acc), 0, abort_flag, g.status);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int t2 = 0; t2 < (two ? 2 : 1); ++t2) {
+            const int tile = tile0 + t2;
+            const int n = tile * kWeightTileRows + lg * 32 + lane;
+            const uint32_t taddr = tmem_d + (uint32_t)(256 * t2) + ((uint32_t)(lg * 32) << 16);
+            if (ok && nkb > 0) {
+                for (int c0 = 0; c0 < g.rows; c0 += 8) {
+                    float v[8];
+                    tmem_ld8(taddr + (uint32_t)c0, v);
+                    if (!g.head) {
+                        if (n < g.N) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if (c0 + i < g.rows) g.part[sp * g.split_stride + (size_t)(g.row0 + c0 + i) * g.N + n] = v[i];
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (c0 + i >= g.rows) break;   // uniform across the warp
+                            const int t = g.row0 + c0 + i;
+                            const float val = (n < g.N) ? v[i] : -INFINITY;
+                            if (g.logits && n < g.N) {
+                                const int b = t / g.R_pad, j = t % g.R_pad;
+                                if (j < g.n_rows[b]) g.logits[((size_t)b * g.max_rows + j) * g.N + n] = val;
+                            }
+                            const Top2 best = top2_warp(Top2{val, -INFINITY, n < g.N ? n : 0x7fffffff});
+                            if (lane == 0) {
+                                float *o = g.top_part + ((size_t)(tile * 4 + lg) * g.T_pad + t) * 4;
+                                o[0] = best.v1; o[1] = __int_as_float(best.i1); o[2] = best.v2;
+                            }
+                        }
+                    }
+                }
+            } else if (ok && !g.head) {   // empty split: contributes zeros
+                if (n < g.N)
+                    for (int c = 0; c < g.rows; ++c) g.part[sp * g.split_stride + (size_t)(g.row0 + c) * g.N + n] = 0.0f;
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (s_abort && threadIdx.x == 0) {
+        for (int s = 0; s < g.stages && s < nkb; ++s)
+            for (uint32_t it = 0; it < (1u << 16); ++it)
+                if (mbar_try_wait(smem_u32(&bar_full[s]), 0) || mbar_try_wait(smem_u32(&bar_full[s]), 1)) break;
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(512u) : "memory");
+    }
+}
+
 }  // namespace hispec

@@ -356,6 +356,7 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
     CKB(cudaMemcpy(c->inv_freq, f, sizeof(double) * half, cudaMemcpyHostToDevice));
     delete[] f;
     CKB(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
+    CKB(cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
     CKB(cudaMemset(c->ext.bar, 0, 2 * sizeof(unsigned)));
     CKB(cudaMemcpy(c->ext.d_attn_norm, c->attn_norm, sizeof(float *) * L, cudaMemcpyHostToDevice));
     CKB(cudaMemcpy(c->ext.d_ffn_norm, c->ffn_norm, sizeof(float *) * L, cudaMemcpyHostToDevice));
@@ -567,8 +568,9 @@ struct StageCall {
 };
 
 // one projection: activation buffer `which` (0: act_d, 1: act_o, 2: act_f) times weight matrix
+// *splits_used (may be NULL) receives the number of split-K partial slots written per output element
 int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const CUtensorMap *tmW, int which,
-             int T_pad, const StageCall &sc) {
+             int T_pad, const StageCall &sc, int *splits_used = nullptr) {
     const GemmPlan &p = c->plan[kind];
     hispec_ctx_ext *x = ext_of(c);
     const bool plain = (c->d.flags & HISPEC_FLAG_PLAIN_ACT) != 0;
@@ -578,6 +580,22 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
     const bool head = kind == G_HEAD;
     const size_t split_stride = (size_t)T_pad * p.N;
     if (!head && (size_t)p.splits * split_stride > c->part_floats) return HISPEC_ECAPACITY;
+    // More than 64 rows: two weight tiles per CTA share an activation tile (gemm_pair_kernel), one CTA per SM;
+    // the K range is split so that the grid still fills the GPU once.
+    // (only while three stages of two weight tiles + the activation tile fit: up to 160 rows with hi/lo planes)
+    const int pair_rows = T_pad < 256 ? T_pad : 256;
+    const bool pair_mode = !simt && T_pad > 64 &&
+                           3 * (2 * kWTileBytes + round_up(pair_rows, 16) * planes * 128) + 1024 <= kGemmMaxDynSmem;
+    int splits = head ? 1 : p.splits;
+    if (pair_mode && !head) {
+        const int pairs = ceil_div(p.tiles, 2);
+        splits = (c->sm_count + pairs / 2) / pairs;
+        if (splits < 1) splits = 1;
+        if (splits > kMaxSplits) splits = kMaxSplits;
+        if (splits > p.kb_total / 4) splits = p.kb_total / 4 > 0 ? p.kb_total / 4 : 1;
+        while (splits > 1 && (size_t)splits * split_stride > c->part_floats) --splits;
+    }
+    if (splits_used) *splits_used = splits;
     const int chunk = 256;   // rows one launch can take (with hi/lo planes beyond 128 rows: one MMA per plane)
     for (int row0 = 0; row0 < T_pad; row0 += chunk) {
         int rows = T_pad - row0 < chunk ? T_pad - row0 : chunk;
@@ -598,9 +616,29 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
         }
         GemmArgs g;
         memset(&g, 0, sizeof(g));
-        g.N = p.N; g.K = p.K; g.kb_total = p.kb_total; g.splits = head ? 1 : p.splits;
+        g.N = p.N; g.K = p.K; g.kb_total = p.kb_total; g.splits = splits;
         g.row0 = row0; g.rows = rows;
         g.planes = planes;
+        if (pair_mode) {
+            g.t_box = round_up(rows, 16);
+            const int stage_bytes = 2 * kWTileBytes + g.t_box * planes * 128;
+            int stages = (kGemmMaxDynSmem - 1024) / stage_bytes;
+            if (stages < 2) return HISPEC_ECAPACITY;
+            if (stages > 16) stages = 16;
+            g.stages = stages;
+            g.tmem_cols = 512;
+            g.head = head ? 1 : 0;
+            g.part = c->part; g.split_stride = split_stride;
+            g.top_part = c->top_part; g.T_pad = T_pad;
+            g.logits = (head && sc.res) ? sc.res->logits : nullptr;
+            g.R_pad = sc.a.R_pad; g.max_rows = sc.a.max_rows; g.n_rows = c->rows.n_rows;
+            g.status = c->status;
+            const CUtensorMap *tmXp = act_map(c, which, act, p.K, g.t_box, planes);
+            if (!tmXp || !tmW) return HISPEC_ECUDA;
+            CK(launch(c, st, gemm_pair_kernel, dim3(ceil_div(p.tiles, 2), splits), dim3(kGemmThreads),
+                      (size_t)stages * stage_bytes + 1024, *tmW, *tmXp, g));
+            continue;
+        }
         g.split_planes = (planes == 2 && rows > 128) ? 1 : 0;
         g.t_box = round_up(rows, (planes == 2 && !g.split_planes) ? 8 : 16);
         int ncols = g.t_box * planes;
@@ -809,8 +847,8 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         const int pool_layer = l - kv.first_layer;
         int rc;
         const GemmPlan &pq = c->plan[G_QKV], &po = c->plan[G_O], &pg = c->plan[G_GU], &pd = c->plan[G_DOWN];
-        int sq = simt ? pq.splits : pq.splits;
-        if ((rc = run_gemm(c, st, G_QKV, c->wqkv[l], &c->tm_wqkv[l], 0, T_pad, sc)) != 0) return rc;
+        int sq = pq.splits, so = po.splits, sg = pg.splits, sd = pd.splits;
+        if ((rc = run_gemm(c, st, G_QKV, c->wqkv[l], &c->tm_wqkv[l], 0, T_pad, sc, &sq)) != 0) return rc;
         CK(launch(c, st, qkv_rope_store_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, sq,
                   (size_t)T_pad * pq.N, d.n_q_heads, d.n_kv_heads, d.head_dim, (const double *)c->inv_freq, c->q,
                   (__nv_bfloat16 *)kv.k_pages, (__nv_bfloat16 *)kv.v_pages, kv.block_table, (long long)kv.n_pages,
@@ -854,17 +892,17 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
                           (const float *)c->attn_part, ta.n_splits, d.n_q_heads, c->act_o, x->T_alloc, plain));
             }
         }
-        if ((rc = run_gemm(c, st, G_O, c->wo[l], &c->tm_wo[l], 1, T_pad, sc)) != 0) return rc;
-        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, po.splits,
+        if ((rc = run_gemm(c, st, G_O, c->wo[l], &c->tm_wo[l], 1, T_pad, sc, &so)) != 0) return rc;
+        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, so,
                   (size_t)T_pad * po.N, c->ffn_norm[l], d.rms_eps, d.d_model, c->x, c->act_d, x->T_alloc, plain,
                   (float *)nullptr, (float *)nullptr));
-        if ((rc = run_gemm(c, st, G_GU, c->wgu[l], &c->tm_wgu[l], 0, T_pad, sc)) != 0) return rc;
+        if ((rc = run_gemm(c, st, G_GU, c->wgu[l], &c->tm_wgu[l], 0, T_pad, sc, &sg)) != 0) return rc;
         CK(launch(c, st, silu_mul_kernel, dim3(ceil_div(d.d_ffn, 256), T_pad), dim3(256), 0, (const float *)c->part,
-                  pg.splits, (size_t)T_pad * pg.N, d.d_ffn, c->act_f, x->T_alloc, plain));
-        if ((rc = run_gemm(c, st, G_DOWN, c->wdown[l], &c->tm_wdown[l], 2, T_pad, sc)) != 0) return rc;
+                  sg, (size_t)T_pad * pg.N, d.d_ffn, c->act_f, x->T_alloc, plain));
+        if ((rc = run_gemm(c, st, G_DOWN, c->wdown[l], &c->tm_wdown[l], 2, T_pad, sc, &sd)) != 0) return rc;
         const bool last = (l + 1 == a.l1);
         const float *gain = last ? c->final_norm : c->attn_norm[l + 1];
-        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, pd.splits,
+        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, sd,
                   (size_t)T_pad * pd.N, gain, d.rms_eps, d.d_model, c->x, c->act_d, x->T_alloc, plain,
                   last ? exit_buf : (float *)nullptr, last ? hidden_out : (float *)nullptr));
     }
