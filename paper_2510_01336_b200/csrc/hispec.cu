@@ -580,11 +580,12 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
     const bool head = kind == G_HEAD;
     const size_t split_stride = (size_t)T_pad * p.N;
     if (!head && (size_t)p.splits * split_stride > c->part_floats) return HISPEC_ECAPACITY;
-    // More than 64 rows: two weight tiles per CTA share an activation tile (gemm_pair_kernel), one CTA per SM;
-    // the K range is split so that the grid still fills the GPU once.
-    // (only while three stages of two weight tiles + the activation tile fit: up to 160 rows with hi/lo planes)
+    // Between 129 and 160 rows with hi/lo planes (a serving batch of 16 with k = 8): two weight tiles per CTA share
+    // an activation tile (gemm_pair_kernel), one CTA per SM; the K range is split so that the grid still fills the
+    // GPU once.  Up to 128 rows the one-tile kernel (one MMA over both planes, two CTAs per SM) measured 2 % faster;
+    // above 160 rows three stages of the pair no longer fit and it measured 4 % slower.
     const int pair_rows = T_pad < 256 ? T_pad : 256;
-    const bool pair_mode = !simt && T_pad > 64 &&
+    const bool pair_mode = !simt && planes == 2 && T_pad > 128 &&
                            3 * (2 * kWTileBytes + round_up(pair_rows, 16) * planes * 128) + 1024 <= kGemmMaxDynSmem;
     int splits = head ? 1 : p.splits;
     if (pair_mode && !head) {
