@@ -373,8 +373,8 @@ extern "C" int hispec_create(const hispec_model_desc *desc, const hispec_weights
             }
         }
         CKB(cudaMemcpy(c->ext.d_gemms, hg.data(), sizeof(MegaGemm) * hg.size(), cudaMemcpyHostToDevice));
-        CKB(cudaFuncSetAttribute(hispec_stage_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
-        CKB(cudaFuncSetAttribute(hispec_stage_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmMaxDynSmem));
+        CKB(cudaFuncSetAttribute(hispec_stage_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMegaMaxDynSmem));
+        CKB(cudaFuncSetAttribute(hispec_stage_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMegaMaxDynSmem));
         int coop = 0;
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
         c->ext.mega_ok = coop != 0 && d.page_size == 16 && d.max_batch <= kMegaMaxBatch &&
@@ -720,7 +720,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     const int ncols = m.t_box * planes;
     const int attn_bytes = kMegaAttnStages * 2 * 16 * d.head_dim * 2;
     const int stage_bytes = kWTileBytes + ncols * 128;
-    int stages = (kGemmMaxDynSmem - attn_bytes - 1024) / (2 * stage_bytes);  // two pipelines
+    int stages = (kMegaMaxDynSmem - attn_bytes - 1024) / (2 * stage_bytes);  // two pipelines
     // Four stages per pipeline: three cost 2 % (less of the next projection prefetched while the grid waits), five
     // and more cost 1 % (the longer burst of prefetch loads at the end of a projection delays the latency-bound
     // element-wise phase that runs beside it) -- measured on the Llama-3-8B shape, kernel time +-0.1 %.
@@ -731,6 +731,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     m.stages = stages;
     for (int k = 0; k < G_HEAD; ++k) {
         if (x->mega_part_floats[k] * (size_t)T_pad > c->part_floats) return 1;
+        if (c->plan[k].tiles > kMegaSlotTiles) return 1;   // the kernel tabulates the partial-slot range of every tile
         // the kernel's partition arithmetic is 32-bit and its per-pipeline segment lists are fixed-size
         if ((long long)c->plan[k].tiles * c->plan[k].kb_total * 2 * c->sm_count >= (1ll << 31)) return 1;
         if (ceil_div(ceil_div(c->plan[k].tiles * c->plan[k].kb_total, 2 * c->sm_count), c->plan[k].kb_total) + 2 > kMegaMaxSegs) return 1;

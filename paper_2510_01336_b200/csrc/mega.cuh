@@ -51,6 +51,8 @@ constexpr int kWarpMma0 = 1, kWarpX = 3, kWarpEpi0 = 4;
 constexpr int kMegaAccCols = 128;  // TMEM columns per accumulator buffer (2 pipelines x 2 buffers)
 constexpr int kEwChunk = 256;      // columns per element-wise work item (one warp, 8 per lane)
 constexpr int kSsqChunk = 128;     // columns per sum-of-squares record
+constexpr int kMegaMaxDynSmem = 212 * 1024;   // dynamic shared memory of the kernel: 227 KB per CTA less its static tables
+constexpr int kMegaSlotTiles = 512; // output tiles per projection whose partial-slot ranges are tabulated in shared memory
 
 struct __align__(64) MegaGemm {
     CUtensorMap tmW;
@@ -118,6 +120,10 @@ struct MegaShared {
     int abort_flag;
     int trace_n;
     int bar_k;
+    // per output tile of the four layer projections: number of partial slots and the first pipeline that holds one
+    // (worked out once: two divisions per look-up otherwise, in front of every element-wise item's loads)
+    unsigned short slot_n[4][kMegaSlotTiles];
+    unsigned short slot_first[4][kMegaSlotTiles];
     int stamp_on, stamp_n;   // HISPEC_STAMPS builds only: fine-grained time stamps of one layer
     int p0[kMegaMaxBatch], nr[kMegaMaxBatch], nd[kMegaMaxBatch], dst[kMegaMaxBatch];
     float red_v1[8], red_v2[8];
@@ -314,10 +320,9 @@ __device__ __forceinline__ void store8_hilo(__nv_bfloat16 *hi, __nv_bfloat16 *lo
 
 // sum of the split-K partial slots of 8 consecutive columns (all inside one tile), slot order
 // part 0 / 1 of `parts` = 2 takes the first ceil(ns / 2) / the remaining slots (parts = 1: all of them)
-__device__ __forceinline__ void sum_slots8(const MegaArgs &m, const MegaGemm &g, int t, int n, float *v, int part = 0,
-                                           int parts = 1) {
-    int first, ns;
-    mega_slots(n / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
+__device__ __forceinline__ void sum_slots8(const MegaArgs &m, const MegaShared &sh, int kind, const MegaGemm &g, int t, int n,
+                                           float *v, int part = 0, int parts = 1) {
+    int ns = sh.slot_n[kind][n / kWeightTileRows];
     const size_t stride = (size_t)m.T_pad * g.N;
     const float *p = m.part + (size_t)t * g.N + n;
     if (parts == 2) {
@@ -343,9 +348,8 @@ __device__ __forceinline__ void sum_slots8(const MegaArgs &m, const MegaGemm &g,
             }
     }
 }
-__device__ __forceinline__ float sum_slots1(const MegaArgs &m, const MegaGemm &g, int t, int n) {
-    int first, ns;
-    mega_slots(n / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
+__device__ __forceinline__ float sum_slots1(const MegaArgs &m, const MegaShared &sh, int kind, const MegaGemm &g, int t, int n) {
+    const int ns = sh.slot_n[kind][n / kWeightTileRows];
     const size_t stride = (size_t)m.T_pad * g.N;
     const float *p = m.part + (size_t)t * g.N + n;
     float v = 0.f;
@@ -417,7 +421,7 @@ __device__ void ew_rope_table(const MegaArgs &m, MegaShared &sh, int gw, int ngw
 }
 
 // a5/a7 epilogue: x += projection; act_d <- hi/lo(x .* gain); chunk sums of squares; exit rows on the last layer
-__device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, const float *gain, float *exit_buf,
+__device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int kind, const float *gain, float *exit_buf,
                          float *hidden_out, int gw, int ngw, int lane) {
     // One warp per (row, 128 columns): the half-warps each add half of the partial slots (a tile of O or
     // down has about ten), 8 columns per lane, and exchange their sums; then half 0 stores the fp32 row,
@@ -440,7 +444,7 @@ __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, c
             q = *reinterpret_cast<const float4 *>(xr + 4);
             g0 = *reinterpret_cast<const float4 *>(gain + c);   // fetched with everything else: the gain vector of a
             g1 = *reinterpret_cast<const float4 *>(gain + c + 4);   // layer is cold, one more round trip if loaded at its use
-            sum_slots8(m, g, t, c, v, hl, 2);
+            sum_slots8(m, sh, kind, g, t, c, v, hl, 2);
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -519,8 +523,7 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         // must not wait for this load's round trip
         const long long page = m.block_table[(size_t)b * a.max_pages + lp];
         // a head's columns lie in one 128-row weight tile (head_dim 64 or 128): one slot range for the item
-        int first, ns;
-        mega_slots((h * hd) / kWeightTileRows, g.tiles, g.kb_total, gridDim.x, first, ns);
+        const int ns = sh.slot_n[0][(h * hd) / kWeightTileRows];
         const float *pr = m.part + (size_t)t * g.N + h * hd;
         // lane l owns columns l + 32 e of the head (e < hd / 32; hd is 64 or 128).  Every load of the item --
         // chunk sums, rotary pair, up to eight slots of each column -- is issued before the first use.
@@ -583,7 +586,7 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
 }
 
 // a6 epilogue: act_f <- hi/lo( SiLU(gate / rms) * (up / rms) )
-__device__ void ew_silu(const MegaArgs &m, const MegaGemm &g, int gw, int ngw, int lane) {
+__device__ void ew_silu(const MegaArgs &m, const MegaShared &sh, const MegaGemm &g, int gw, int ngw, int lane) {
     const int nch = (m.ffn + kEwChunk - 1) / kEwChunk;
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
         const int t = item / nch, ch = item % nch;
@@ -591,8 +594,8 @@ __device__ void ew_silu(const MegaArgs &m, const MegaGemm &g, int gw, int ngw, i
         const float ssq = mega_ssq_fetch(m, t, lane);
         float gt[8], up[8], v[8];
         if (c < m.ffn) {
-            sum_slots8(m, g, t, c, gt);
-            sum_slots8(m, g, t, m.ffn + c, up);
+            sum_slots8(m, sh, 2, g, t, c, gt);
+            sum_slots8(m, sh, 2, g, t, m.ffn + c, up);
         }
         const float inv = mega_inv_rms_finish(m, ssq);
         if (c >= m.ffn) continue;
@@ -1089,9 +1092,7 @@ __device__ __forceinline__ bool mega_epilogue_part(const MegaGemm *g, int kind, 
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = sh.tmem + (p * 2 + buf) * kMegaAccCols + ((uint32_t)(lg * 32) << 16);
             const int n = tile * kWeightTileRows + lg * 32 + lane;
-            int first, ns;
-            mega_slots(tile, g->tiles, g->kb_total, gridDim.x, first, ns);
-            const int slot = 2 * blockIdx.x + p - first;
+            const int slot = 2 * blockIdx.x + p - (int)sh.slot_first[kind][tile];
             for (int c0 = 0; c0 < m.T_pad; c0 += 8) {
                 float v[8];
                 mega_acc_ld8(taddr, c0, m.t_box, m.planes, v);
@@ -1321,6 +1322,16 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
     }
     mega_prep_rows(m, sh, 0, threadIdx.x, blockDim.x);
     mega_fill_seglists(m, sh);
+    for (int i = threadIdx.x; i < 4 * kMegaSlotTiles; i += blockDim.x) {
+        const int kind = i / kMegaSlotTiles, tile = i % kMegaSlotTiles;
+        const MegaGemm &g = m.gemms[m.a.l0 * 4 + kind];
+        if (tile < g.tiles) {
+            int first, ns;
+            mega_slots(tile, g.tiles, g.kb_total, gridDim.x, first, ns);
+            sh.slot_n[kind][tile] = (unsigned short)ns;
+            sh.slot_first[kind][tile] = (unsigned short)first;
+        }
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1382,13 +1393,13 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
                     ew_attn_merge<HD>(m, sh, gw, ngw, lane);
                 } else if (kind == 2) {
                     MEGA_STAMP(74);
-                    ew_silu(m, G4[2], gw, ngw, lane);
+                    ew_silu(m, sh, G4[2], gw, ngw, lane);
                     MEGA_STAMP(75);
                 } else {
                     const bool last = kind == 3 && l + 1 == a.l1;
                     const float *gain = kind == 1 ? m.ffn_norm[l] : (last ? m.final_norm : m.attn_norm[l + 1]);
                     MEGA_STAMP(72);
-                    ew_resid(m, sh, G4[kind], gain, last ? m.exit_buf : nullptr, last ? m.hidden_out : nullptr, gw, ngw, lane);
+                    ew_resid(m, sh, G4[kind], kind, gain, last ? m.exit_buf : nullptr, last ? m.hidden_out : nullptr, gw, ngw, lane);
                     MEGA_STAMP(73);
                 }
                 grid_sync(m, sh);
