@@ -397,6 +397,65 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_configs(args):
+    """The two serving configurations of the workload list beside the benchmarked one: per-call latency of the
+    intermediate and the target verification on seeded random state (median of 15 calls), with the algorithmic
+    bytes and flops of each call.  cfg3: Llama-3-8B shape, 16 sequences, contexts uniform in [512, 4096], k = 8
+    (9 rows with the bonus row; the target checks 2 x 9 = 18 rows).  cfg4: Llama-2-13B shape, 8 sequences, context
+    2048, k = 6 (7 rows; target 14).  One JSON line per call (not the benchmark line)."""
+    import torch
+    from paper_2510_01336_b200 import binding, workload as wl
+    torch.cuda.set_device(0)
+    peak, _ = peaks()
+    cases = [("cfg3", wl.L3_8B, 16, 8, wl.make_prompt_lengths(wl.L3_8B, 16, 512, 4096)),
+             ("cfg4", wl.L2_13B, 8, 6, [2048] * 8)]
+    for name, shape, B, k, ctx_lens in cases:
+        for call, l0, l1, R in (("verify_i", shape.L_d, shape.L_i, k + 1), ("verify_t", shape.L_i, shape.L_f, 2 * (k + 1))):
+            layers = list(range(l0, l1))
+            w = wl.make_weights(shape, layers=layers, device="cuda", with_emb=False)
+            max_rows = 2 * (k + 1) + 1
+            max_pages = (max(ctx_lens) + max_rows + 15) // 16 + 1
+            ctxo = binding.Context(shape, w, page_size=16, max_batch=B, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+            st = ctxo.new_state(B, B * max_pages, wl.make_block_table(shape, B, max_pages), first_layer=l0,
+                                n_pool_layers=len(layers))
+            g = torch.Generator(device="cuda").manual_seed(shape.seed + 4000)
+            for t in (st.k_pages, st.v_pages, st.h_draft, st.h_inter):
+                t.normal_(generator=g)
+            res = ctxo.new_result(B)
+            base = torch.tensor(ctx_lens, dtype=torch.int32, device="cuda")
+            drafts = torch.zeros((B, max_rows - 1), dtype=torch.int32, device="cuda")
+            nr = torch.full((B,), R, dtype=torch.int32, device="cuda")
+            nd = torch.full((B,), R - 1 if call == "verify_i" else R, dtype=torch.int32, device="cuda")
+            times = []
+            for it in range(18):
+                st.len_draft.copy_(base + R)
+                st.len_inter.copy_(base + (R if call == "verify_t" else 0))
+                st.len_target.copy_(base)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                # k of the call: rows are padded to k + 1 per sequence, so the tightest k that admits the rows
+                (ctxo.verify_intermediate if call == "verify_i" else ctxo.verify_target)(st, drafts, nd, nr, res, k=R - 1 if call == "verify_i" else R)
+                e1.record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    times.append(e0.elapsed_time(e1))
+            times.sort()
+            ms = times[len(times) // 2]
+            T = B * R
+            by = (len(layers) * shape.layer_weight_bytes + shape.head_bytes +
+                  sum(len(layers) * shape.kv_bytes_per_token_layer * (c + R) for c in ctx_lens) + 2 * T * shape.d_model * 4)
+            fl = 2.0 * T * (len(layers) * shape.layer_params + shape.vocab * shape.d_model) + \
+                sum(len(layers) * 4.0 * shape.n_q_heads * shape.head_dim * R * (c + (R + 1) / 2) for c in ctx_lens)
+            print(json.dumps({"config": name, "shape": shape.name, "call": call, "layers": [l0, l1], "batch": B, "rows_per_seq": R,
+                              "mean_ctx": round(sum(ctx_lens) / B), "us": round(ms * 1e3, 1),
+                              "algorithmic_gb": round(by / 1e9, 3), "gbs": round(by / ms / 1e6, 0),
+                              "frac_of_measured_hbm": round(by / ms / 1e6 / peak, 3), "tflops": round(fl / ms / 1e9, 1),
+                              "status": ctxo.status()}), flush=True)
+            ctxo.close()
+            del st, ctxo, w
+            torch.cuda.empty_cache()
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
@@ -426,6 +485,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the AR / Algorithm 1 / acceptance-shaped context numbers")
     ap.add_argument("--sweep", action="store_true", help="verify-step latency vs k / batch / context (not the bench line)")
     ap.add_argument("--sweep-all-li", action="store_true", help="sweep intermediate exits 12, 16, 24 instead of 16 only")
+    ap.add_argument("--configs", action="store_true", help="per-call latency of the serving configurations cfg3 / cfg4 (not the bench line)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -433,6 +493,9 @@ def main():
     if args.sweep:
         if rank == 0:
             run_sweep(args)
+    elif args.configs:
+        if rank == 0:
+            run_configs(args)
     elif args.impl == "reference":
         run_reference(args, rank, world)
     else:

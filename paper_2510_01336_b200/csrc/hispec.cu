@@ -718,8 +718,10 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     m.T_pad = T_pad; m.T_alloc = x->T_alloc; m.planes = planes; m.plain = plain;
     m.t_box = round_up(T_pad, planes == 2 ? 8 : 16);
     const int ncols = m.t_box * planes;
-    const int attn_bytes = kMegaAttnStages * 2 * 16 * d.head_dim * 2;
     const int stage_bytes = kWTileBytes + ncols * 128;
+    // with at least 8 KB of activation tile per stage the attention phase borrows those areas for its KV pages
+    m.attn_in_ring = (ncols * 128 >= 2 * 16 * d.head_dim * 2 && kMegaAttnStages <= 4) ? 1 : 0;
+    const int attn_bytes = m.attn_in_ring ? 0 : kMegaAttnStages * 2 * 16 * d.head_dim * 2;
     int stages = (kMegaMaxDynSmem - attn_bytes - 1024) / (2 * stage_bytes);  // two pipelines
     // Four stages per pipeline: three cost 2 % (less of the next projection prefetched while the grid waits), five
     // and more cost 1 % (the longer burst of prefetch loads at the end of a projection delays the latency-bound

@@ -84,6 +84,7 @@ struct MegaArgs {
     float *q, *part, *attn_part, *top_part, *ssq;
     // a block of draft steps in one launch (hispec_draft_block): the call's steps a0..a10 run n_rep times; step s > 0
     // reads its token from block[b * block_stride + s - 1], step s < n_steps writes block[b * block_stride + s]
+    int attn_in_ring;        // the attention phase stages its KV pages in the activation areas of the ring stages
     int n_rep, n_steps, block_stride;
     int32_t *block;
     float *cta_top;          // [gridDim.x][T_pad][4]: each CTA's top-2 over its own exit-head tiles (v1, id1, v2, -)
@@ -676,10 +677,16 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
     MEGA_STAMP(32);
 }
 
+// shared-memory address of KV page stage s (s < 4): a0 + (s & 1) * d1 + (s >> 1) * d2
+struct AttnSmem {
+    uint32_t a0, d1, d2;
+    __device__ __forceinline__ uint32_t at(int s) const { return a0 + (uint32_t)(s & 1) * d1 + (uint32_t)(s >> 1) * d2; }
+};
+
 // ---- attention phase: items (split, kv head x row group, sequence) dealt round-robin to CTAs -------
 template <int HD>
 __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, const MegaArgs &m, MegaShared &sh,
-                               uint32_t sm_attn, int pool_layer, uint32_t &pg_it, int warp, int lane) {
+                               const AttnSmem sm_attn, int pool_layer, uint32_t &pg_it, int warp, int lane) {
     constexpr int HALVES = HD / 64, TILE = 16 * HD * 2, KS = HD / 16, NT = HD / 8;
     const StageArgs &a = m.a;
     volatile int *abort_flag = &sh.abort_flag;
@@ -713,7 +720,7 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                         const uint32_t fb = a_smem_u32(&sh.a_full[s]);
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(2 * TILE) : "memory");
                         const int row = (int)((((long long)pool_layer * m.n_pages + page) * m.hkv + kvh) * 16);
-                        const uint32_t dk = sm_attn + s * 2 * TILE, dv = dk + TILE;
+                        const uint32_t dk = sm_attn.at(s), dv = dk + TILE;
 #pragma unroll
                         for (int h = 0; h < HALVES; ++h) {
                             tma_load_2d(dk + h * 2048, tmK, h * 64, row, fb);
@@ -768,7 +775,7 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                 if (!ok) break;
                 MEGA_STAMP(22);
                 if (active && (i % m.ngrp) == grp) {
-                    const uint32_t sk = sm_attn + s * 2 * TILE, sv = sk + TILE;
+                    const uint32_t sk = sm_attn.at(s), sv = sk + TILE;
                     // four independent accumulator chains (2 key tiles x hi/lo query planes), added at the end
                     float sc[2][4], sl[2][4];
 #pragma unroll
@@ -1285,7 +1292,15 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         ring[p].stages = m.stages;
         ring[p].base = base + p * m.stages * ring[p].stage_bytes;
     }
-    const uint32_t sm_attn = base + 2 * m.stages * ring[0].stage_bytes;  // 1024-aligned: stage_bytes is a multiple of 2048
+    // KV page staging of the attention phase: its own area behind the rings, or -- with many rows, where an
+    // activation tile is at least as large as a K + V page -- the activation areas of four ring stages, which are
+    // idle between two projections (that shared memory then buys another ring stage)
+    AttnSmem sm_attn;
+    if (m.attn_in_ring) {
+        sm_attn.a0 = ring[0].base + kWTileBytes; sm_attn.d1 = ring[1].base - ring[0].base; sm_attn.d2 = ring[0].stage_bytes;
+    } else {
+        sm_attn.a0 = base + 2 * m.stages * ring[0].stage_bytes; sm_attn.d1 = 2 * 16 * HD * 2; sm_attn.d2 = 2 * sm_attn.d1;
+    }
 
     if (threadIdx.x == 0) {
         sh.abort_flag = 0;
