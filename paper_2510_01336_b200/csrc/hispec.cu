@@ -50,6 +50,19 @@ bool encode_2d(CUtensorMap *tm, const void *base, uint64_t K, uint64_t rows, uin
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// KV pages for the persistent kernel: [rows][halves][64] with the halves as the outermost box dimension
+bool encode_pages3(CUtensorMap *tm, const void *base, uint64_t hd, uint64_t rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kTileK, rows, hd / kTileK};
+    cuuint64_t strides[2] = {hd * 2, (cuuint64_t)kTileK * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kTileK, 16, (cuuint32_t)(hd / kTileK)};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // activation buffer [2 planes][T_alloc][K]
 bool encode_act(CUtensorMap *tm, const void *base, uint64_t K, uint64_t T_alloc, uint32_t t_box, uint32_t planes) {
     EncodeTiledFn fn = get_encode_fn();
@@ -112,7 +125,9 @@ struct hispec_ctx_ext {
     bool profiling;
     std::vector<ProfEvent> *prof;       // recorded since the last read
     std::vector<ProfEvent> *prof_free;  // event pairs ready for reuse
-    struct PageMaps { const void *k, *v; long long n_pages; int pool_layers; CUtensorMap tmK, tmV; } page_maps[4];
+    // tmK / tmV: rows of head_dim elements, box 64 x 16; tmK3 / tmV3: the same pages with the head dimension seen as
+    // [head_dim / 64][64], box 64 x 16 x (head_dim / 64): a whole K (or V) page of one KV head in one TMA copy
+    struct PageMaps { const void *k, *v; long long n_pages; int pool_layers; CUtensorMap tmK, tmV, tmK3, tmV3; } page_maps[4];
     int n_page_maps;
     ActMapCache act_cache[3][8];
     int act_cache_n[3];
@@ -534,7 +549,8 @@ const hispec_ctx_ext::PageMaps *page_maps(hispec_ctx *c, const hispec_kv &kv) {
     int slot = x->n_page_maps < 4 ? x->n_page_maps++ : 3;
     auto &m = x->page_maps[slot];
     uint64_t rows = (uint64_t)kv.n_pool_layers * kv.n_pages * c->d.n_kv_heads * c->d.page_size;
-    if (!encode_2d(&m.tmK, kv.k_pages, c->d.head_dim, rows, 16) || !encode_2d(&m.tmV, kv.v_pages, c->d.head_dim, rows, 16)) {
+    if (!encode_2d(&m.tmK, kv.k_pages, c->d.head_dim, rows, 16) || !encode_2d(&m.tmV, kv.v_pages, c->d.head_dim, rows, 16) ||
+        !encode_pages3(&m.tmK3, kv.k_pages, c->d.head_dim, rows) || !encode_pages3(&m.tmV3, kv.v_pages, c->d.head_dim, rows)) {
         x->n_page_maps = slot;
         return nullptr;
     }
@@ -695,15 +711,13 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     const int planes = plain ? 1 : 2;
     if (!x->mega_ok || T_pad * planes > kMegaAccCols) return 1;
     const hispec_kv &kv = *sc.kv;
-    {
-        // The persistent kernel is built for calls dominated by the weight stream.  When the KV cache
-        // a layer may have to read (by the block-table capacity; the lengths live on the device) outweighs
-        // the layer's weights, the stand-alone attention kernel with its deeper page pipeline serves better.
-        double kv_cap = (double)a.batch * d.max_pages_per_seq * d.page_size * 4.0 * d.n_kv_heads * d.head_dim;
-        double w_layer = 0.0;
-        for (int k = 0; k < G_HEAD; ++k) w_layer += 2.0 * (double)c->plan[k].N * c->plan[k].K;
-        if (kv_cap > w_layer && !env_int("HISPEC_FORCE_MEGA", 0)) return 1;
-    }
+    // The persistent kernel is built for calls dominated by the weight stream.  When the KV cache
+    // a layer may have to read (by the block-table capacity; the lengths live on the device) outweighs
+    // the layer's weights, the stand-alone attention kernel with its deeper page pipeline serves better.
+    const double kv_cap = (double)a.batch * d.max_pages_per_seq * d.page_size * 4.0 * d.n_kv_heads * d.head_dim;
+    double w_layer = 0.0;
+    for (int k = 0; k < G_HEAD; ++k) w_layer += 2.0 * (double)c->plan[k].N * c->plan[k].K;
+    if (kv_cap > w_layer && !env_int("HISPEC_FORCE_MEGA", 0)) return 1;
     MegaArgs m;
     memset(&m, 0, sizeof(m));
     m.a = a;
@@ -719,17 +733,32 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     m.t_box = round_up(T_pad, planes == 2 ? 8 : 16);
     const int ncols = m.t_box * planes;
     const int stage_bytes = kWTileBytes + ncols * 128;
-    // with at least 8 KB of activation tile per stage the attention phase borrows those areas for its KV pages
-    m.attn_in_ring = (ncols * 128 >= 2 * 16 * d.head_dim * 2 && kMegaAttnStages <= 4) ? 1 : 0;
-    const int attn_bytes = m.attn_in_ring ? 0 : kMegaAttnStages * 2 * 16 * d.head_dim * 2;
-    int stages = (kMegaMaxDynSmem - attn_bytes - 1024) / (2 * stage_bytes);  // two pipelines
-    // Four stages per pipeline: three cost 2 % (less of the next projection prefetched while the grid waits), five
-    // and more cost 1 % (the longer burst of prefetch loads at the end of a projection delays the latency-bound
-    // element-wise phase that runs beside it) -- measured on the Llama-3-8B shape, kernel time +-0.1 %.
-    int cap = env_int("HISPEC_MEGA_STAGES", 4);
+    // Four ring stages per pipeline: three cost 2 % (less of the next projection prefetched while the grid waits),
+    // five and more cost 1 % (the longer burst of prefetch loads at the end of a projection delays the latency-bound
+    // element-wise phase beside it; Llama-3-8B shape, kernel time +-0.1 %).
+    // KV page staging of the attention phase (a K + V page of one KV head is 8 KB at head_dim 128):
+    //  - weight-dominated calls: four pages in flight, in the ring's idle activation areas where those are large
+    //    enough (32 rows and more), else in an area of their own; the weight producer prefetches the output
+    //    projection into the rings meanwhile;
+    //  - calls whose KV cache per layer may reach a tenth of the layer's weights: the attention phase is bound by the
+    //    bytes it has in flight, so it takes both rings whole (up to kMegaAttnStages pages) and the weight producer
+    //    waits for it; the output projection's first blocks then arrive during the split merge.
+    const int page_bytes = 2 * 16 * d.head_dim * 2;
+    const int budget = kMegaMaxDynSmem - 1024;
+    const int cap = env_int("HISPEC_MEGA_STAGES", 4);
+    const bool kv_heavy = kv_cap >= 0.1 * w_layer && !env_int("HISPEC_NO_WIDE", 0);
+    m.attn_in_ring = kv_heavy ? 2 : ((ncols * 128 >= page_bytes) ? 1 : 0);
+    int stages = (budget - (m.attn_in_ring ? 0 : 4 * page_bytes)) / (2 * stage_bytes);
     if (stages > cap) stages = cap;
     if (stages > kMegaMaxStages) stages = kMegaMaxStages;
     if (stages < 2) return 1;
+    m.attn_stages = m.attn_in_ring == 2 ? 2 * stages * stage_bytes / page_bytes : 4;
+    if (m.attn_stages > kMegaAttnStages) m.attn_stages = kMegaAttnStages;
+    // a power of two: the two page producers and the warp groups (1, 2 or 4) divide it, and the kernel shifts and masks
+    m.attn_log2 = 2;
+    while ((2 << m.attn_log2) <= m.attn_stages) ++m.attn_log2;
+    m.attn_stages = 1 << m.attn_log2;
+    const int attn_bytes = m.attn_in_ring ? 0 : 4 * page_bytes;
     m.stages = stages;
     for (int k = 0; k < G_HEAD; ++k) {
         if (x->mega_part_floats[k] * (size_t)T_pad > c->part_floats) return 1;
@@ -764,6 +793,9 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     if (m.n_splits > 16) m.n_splits = 16;
     m.ngrp = m.mt == 1 ? 4 : (m.mt == 2 ? 2 : 1);
     if (m.n_splits * m.ngrp > 32) m.ngrp = 32 / m.n_splits;   // one load batch in the split merge (16 splits: ngrp <= 2)
+    if (m.ngrp == 3) m.ngrp = 2;
+    m.attn_stages -= m.attn_stages % m.ngrp;   // a stage belongs to one warp group
+    if (m.attn_stages < m.ngrp) return 1;
     if ((size_t)m.n_splits * m.ngrp * T_pad * d.n_q_heads * (d.head_dim + kAttnRecPad) > c->attn_part_floats) return 1;
     m.scale_log2 = (1.0f / sqrtf((float)d.head_dim)) * 1.4426950408889634f;
     m.r.len_d = kv.len_draft; m.r.len_i = kv.len_inter; m.r.len_f = kv.len_target;
@@ -806,8 +838,8 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     wbytes *= m.n_rep;
     ProfScope prof(c, st, 20, wbytes);
     cudaError_t le = (d.head_dim == 64)
-                         ? cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m)
-                         : cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m);
+                         ? cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK3, pm->tmV3, m)
+                         : cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK3, pm->tmV3, m);
     if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorLaunchOutOfResources) {
         // the GPU cannot hold one CTA per SM at once (e.g. it is shared): use the kernel sequence from now on
         (void)cudaGetLastError();

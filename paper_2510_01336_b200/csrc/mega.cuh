@@ -40,7 +40,7 @@ namespace hispec {
 // 168 registers, and the spills that caused cost every phase a memory round trip.
 constexpr int kMegaThreads = 256;
 constexpr int kMegaMaxStages = 8;  // per pipeline
-constexpr int kMegaAttnStages = 4; // KV pages in flight per CTA in the attention phase (8 KB each at head_dim 128); 8 measured: +2 % on the 12-row call at context 1024, -2 % at context 16384
+constexpr int kMegaAttnStages = 16; // most KV pages in flight per CTA in the attention phase (8 KB each at head_dim 128); a call uses 4 to 16
 constexpr int kMegaMaxBatch = 64;
 constexpr int kMegaWorkers = 224;  // threads of warps 1..7
 constexpr int kMegaLeader = 32;    // warp 1 lane 0
@@ -84,7 +84,11 @@ struct MegaArgs {
     float *q, *part, *attn_part, *top_part, *ssq;
     // a block of draft steps in one launch (hispec_draft_block): the call's steps a0..a10 run n_rep times; step s > 0
     // reads its token from block[b * block_stride + s - 1], step s < n_steps writes block[b * block_stride + s]
-    int attn_in_ring;        // the attention phase stages its KV pages in the activation areas of the ring stages
+    int attn_log2;           // attn_stages == 1 << attn_log2
+    int attn_stages;         // KV pages in flight per CTA (4 at short contexts: 8 measured +2 % on a 12-row call at context 1024, -2 % at 16384)
+    int attn_in_ring;        // where the attention phase stages its KV pages: 0 an area of its own behind the rings, 1 the activation
+                             // areas of the ring stages, 2 the whole of both rings (the weight producer then holds the output
+                             // projection's blocks back until the CTA's attention items are done)
     int n_rep, n_steps, block_stride;
     int32_t *block;
     float *cta_top;          // [gridDim.x][T_pad][4]: each CTA's top-2 over its own exit-head tiles (v1, id1, v2, -)
@@ -119,6 +123,7 @@ struct MegaShared {
     uint64_t a_full[kMegaAttnStages], a_empty[kMegaAttnStages];
     uint32_t tmem;
     int abort_flag;
+    int attn_epoch;          // attention phases this CTA has finished (attn_in_ring == 2: releases the weight producer)
     int trace_n;
     int bar_k;
     // per output tile of the four layer projections: number of partial slots and the first pipeline that holds one
@@ -677,7 +682,15 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
     MEGA_STAMP(32);
 }
 
-// shared-memory address of KV page stage s (s < 4): a0 + (s & 1) * d1 + (s >> 1) * d2
+// one round of a polling loop that serves several queues with non-blocking tests: bounded, and gives up once the CTA aborts
+__device__ __forceinline__ bool mega_poll_idle(uint32_t &idle, bool did, volatile int *ab, uint32_t *status) {
+    if (did) { idle = 0; return true; }
+    if (++idle >= (1u << 28)) { *ab = 1; atomicOr(status, HISPEC_ST_TIMEOUT); return false; }
+    if ((idle & 65535u) == 0u && *ab) return false;
+    return true;
+}
+
+// shared-memory address of KV page stage s: a0 + (s & 1) * d1 + (s >> 1) * d2
 struct AttnSmem {
     uint32_t a0, d1, d2;
     __device__ __forceinline__ uint32_t at(int s) const { return a0 + (uint32_t)(s & 1) * d1 + (uint32_t)(s >> 1) * d2; }
@@ -703,7 +716,12 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
         if (chunk < 1) chunk = 1;
         const int pg0 = split * chunk, pg1 = min(pg0 + chunk, total_pages);
         const int n_pg = (nr > 0 && pg1 > pg0) ? pg1 - pg0 : 0;
-        if (warp == kWarpX) {
+        if (warp == kWarpX || warp == kWarpMma0 + 1) {
+            // Two page producers -- the activation loader's warp and the second MMA warp, both idle in this phase --
+            // take the pages in turn (the number of stages is even, so a stage always belongs to the same producer):
+            // one issuing thread needs ~0.4 us per page, which bounded the phase on long contexts.  (A producer warp
+            // whose 16 lanes each feed one stage and poll side by side measured 1 to 2 % slower than this.)
+            const uint32_t pw = warp == kWarpX ? 0u : 1u;
             MEGA_STAMP(10);
             for (int i0 = 0; i0 < n_pg; i0 += 32) {
                 const int my = i0 + lane;
@@ -714,18 +732,17 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                 for (int u = 0; u < cnt; ++u) {
                     const long long page = __shfl_sync(0xffffffffu, pgid, u);
                     const uint32_t it = pg_it + i0 + u;
-                    const int s = it % kMegaAttnStages;
-                    const uint32_t ph = (it / kMegaAttnStages) & 1u;
+                    if ((it & 1u) != pw) continue;
+                    const int s = it & (uint32_t)(m.attn_stages - 1);
+                    const uint32_t ph = (it >> m.attn_log2) & 1u;
                     if (lane == 0 && a_wait(a_smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, m.status)) {
                         const uint32_t fb = a_smem_u32(&sh.a_full[s]);
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(2 * TILE) : "memory");
                         const int row = (int)((((long long)pool_layer * m.n_pages + page) * m.hkv + kvh) * 16);
                         const uint32_t dk = sm_attn.at(s), dv = dk + TILE;
-#pragma unroll
-                        for (int h = 0; h < HALVES; ++h) {
-                            tma_load_2d(dk + h * 2048, tmK, h * 64, row, fb);
-                            tma_load_2d(dv + h * 2048, tmV, h * 64, row, fb);
-                        }
+                        // one copy per tensor: the box spans the head dimension's 64-element halves as its third dimension
+                        tma_load_3d(dk, tmK, 0, row, 0, fb);
+                        tma_load_3d(dv, tmV, 0, row, 0, fb);
                     }
                 }
             }
@@ -769,12 +786,15 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             MEGA_STAMP(21);
             for (int i = 0; i < n_pg && ok; ++i) {
                 const uint32_t it = pg_it + i;
-                const int s = it % kMegaAttnStages;
-                const uint32_t ph = (it / kMegaAttnStages) & 1u;
+                // pages go to the warp groups in turn by their running number; the number of stages is a multiple of
+                // the number of groups, so a stage always belongs to the same group and only its warps touch it
+                if ((int)(it % (uint32_t)m.ngrp) != grp) continue;
+                const int s = it & (uint32_t)(m.attn_stages - 1);
+                const uint32_t ph = (it >> m.attn_log2) & 1u;
                 ok = a_wait(a_smem_u32(&sh.a_full[s]), ph, abort_flag, m.status);
                 if (!ok) break;
                 MEGA_STAMP(22);
-                if (active && (i % m.ngrp) == grp) {
+                if (active) {
                     const uint32_t sk = sm_attn.at(s), sv = sk + TILE;
                     // four independent accumulator chains (2 key tiles x hi/lo query planes), added at the end
                     float sc[2][4], sl[2][4];
@@ -933,12 +953,6 @@ struct WCursor {
 // Both polling loops below serve the two pipelines from ONE thread with non-blocking tests: two lanes of a
 // warp that spin in separate loops are not scheduled fairly (one pipeline starves), and a third warp per
 // scheduler partition would cap every thread at 168 registers.
-__device__ __forceinline__ bool mega_poll_idle(uint32_t &idle, bool did, volatile int *ab, uint32_t *status) {
-    if (did) { idle = 0; return true; }
-    if (++idle >= (1u << 28)) { *ab = 1; atomicOr(status, HISPEC_ST_TIMEOUT); return false; }
-    if ((idle & 65535u) == 0u && *ab) return false;
-    return true;
-}
 
 // warp 0, one thread: every weight block of the call, per pipeline in consumption order, into that
 // pipeline's ring -- across projection and phase boundaries.  The first block of a projection is held back
@@ -951,12 +965,24 @@ struct WLane {
     int cur_gi;
     uint32_t last_bar, last_ph;
     bool gate;
-    __device__ WLane(const MegaArgs *m, const MegaShared *sh, int p) : ld(m, sh, p), cur_gi(0), last_bar(0), last_ph(0), gate(false) {
+    int hold;   // attention phases that must have finished before the next block may be loaded (0: none)
+    __device__ WLane(const MegaArgs *m, const MegaShared *sh, int p) : ld(m, sh, p), cur_gi(0), last_bar(0), last_ph(0), gate(false), hold(0) {
         cur_gi = ld.gi;
     }
 };
+// attention phases that precede the projection the cursor stands in (only where the pages take the rings whole;
+// a pipeline without blocks in some projection skips it, so every projection computes its own count)
+__device__ __forceinline__ int mega_w_hold(const MegaArgs &m, const WCursor &c) {
+    if (m.attn_in_ring != 2 || !c.valid) return 0;
+    const int layers = m.a.l1 - m.a.l0, kind = c.kind();
+    return c.rep * layers + (kind == 4 ? layers : (c.gi >> 2) + (kind >= 1 ? 1 : 0));
+}
 __device__ __forceinline__ bool mega_w_issue(const MegaArgs &m, int p, WLane &w, const MegaRing &ring, MegaShared &sh, uint64_t policy) {
     if (!w.ld.valid) return false;
+    if (w.hold) {   // the rings hold KV pages until this CTA's attention items are done
+        if (*((volatile int *)&sh.attn_epoch) < w.hold) return false;
+        w.hold = 0;
+    }
     if (w.gate) {
         if (!mbar_test_wait(w.last_bar, w.last_ph)) return false;
         w.gate = false;
@@ -973,12 +999,18 @@ __device__ __forceinline__ bool mega_w_issue(const MegaArgs &m, int p, WLane &w,
     w.last_ph = w.pos.ph;
     w.ld.advance();
     w.pos.advance(ring.stages);
-    if (w.ld.valid && w.ld.gi + w.ld.rep * w.ld.n_g != w.cur_gi) { w.cur_gi = w.ld.gi + w.ld.rep * w.ld.n_g; w.gate = true; }
+    if (w.ld.valid && w.ld.gi + w.ld.rep * w.ld.n_g != w.cur_gi) {
+        w.cur_gi = w.ld.gi + w.ld.rep * w.ld.n_g;
+        w.gate = true;
+        w.hold = mega_w_hold(m, w.ld);
+    }
     return true;
 }
 __device__ __forceinline__ void mega_w_producer(const MegaArgs &m, const MegaRing *ring, MegaShared &sh) {
     volatile int *ab = &sh.abort_flag;
     WLane w0(&m, &sh, 0), w1(&m, &sh, 1);
+    w0.hold = mega_w_hold(m, w0.ld);
+    w1.hold = mega_w_hold(m, w1.ld);
     // weights are read exactly once per call: mark their lines evict-first so that they do not push the
     // partial sums, activations and KV pages (which are re-read) out of L2
     const uint64_t policy = l2_policy_evict_first();
@@ -1293,10 +1325,12 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         ring[p].base = base + p * m.stages * ring[p].stage_bytes;
     }
     // KV page staging of the attention phase: its own area behind the rings, or -- with many rows, where an
-    // activation tile is at least as large as a K + V page -- the activation areas of four ring stages, which are
+    // activation tile is at least as large as a K + V page -- the activation areas of the ring stages, which are
     // idle between two projections (that shared memory then buys another ring stage)
     AttnSmem sm_attn;
-    if (m.attn_in_ring) {
+    if (m.attn_in_ring == 2) {
+        sm_attn.a0 = base; sm_attn.d1 = 2 * 16 * HD * 2; sm_attn.d2 = 2 * sm_attn.d1;
+    } else if (m.attn_in_ring) {
         sm_attn.a0 = ring[0].base + kWTileBytes; sm_attn.d1 = ring[1].base - ring[0].base; sm_attn.d2 = ring[0].stage_bytes;
     } else {
         sm_attn.a0 = base + 2 * m.stages * ring[0].stage_bytes; sm_attn.d1 = 2 * 16 * HD * 2; sm_attn.d2 = 2 * sm_attn.d1;
@@ -1304,6 +1338,7 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
 
     if (threadIdx.x == 0) {
         sh.abort_flag = 0;
+        sh.attn_epoch = 0;
         sh.trace_n = 0;
         sh.bar_k = 0;
         sh.stamp_on = 0;
@@ -1327,7 +1362,7 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
         }
         for (int s = 0; s < kMegaAttnStages; ++s) {
             mbar_init(smem_u32(&sh.a_full[s]), 1);
-            mbar_init(smem_u32(&sh.a_empty[s]), 4);
+            mbar_init(smem_u32(&sh.a_empty[s]), 4 / m.ngrp);   // the warps of the group that owns the stage
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -1404,6 +1439,10 @@ hispec_stage_kernel(const __grid_constant__ CUtensorMap tmXd, const __grid_const
                     MEGA_STAMP(71);
                     grid_sync(m, sh);
                     mega_attention<HD>(&tmK, &tmV, m, sh, sm_attn, pool_layer, pg_it, warp, lane);
+                    if (m.attn_in_ring == 2) {   // every page has been consumed: the rings go back to the weight producer
+                        worker_bar();
+                        if (threadIdx.x == kMegaLeader) *((volatile int *)&sh.attn_epoch) = sh.attn_epoch + 1;
+                    }
                     grid_sync(m, sh, false);
                     ew_attn_merge<HD>(m, sh, gw, ngw, lane);
                 } else if (kind == 2) {
