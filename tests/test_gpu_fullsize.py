@@ -93,6 +93,15 @@ def test_llama3_8b_shape_serving_batch_ragged():
     _run_case(wl.L3_8B, 8, 16, "verify_i", [517, 1500, 4096], [9, 5, 8], [8, 4, 8], 9, seed_offset=4100)
 
 
+def test_llama3_8b_shape_long_contexts_two_layers():
+    """KV-heavy call (the cache a layer reads is a third of its weights): contexts up to 8192 next to one of a single
+    page, so that the attention phase runs with its deepest page pipeline, several (sequence, KV head, key split)
+    items per CTA and key splits that are empty for the short sequences."""
+    import dataclasses
+    shape = dataclasses.replace(wl.L3_8B, L_d=8, L_i=10, L_f=32)
+    _run_case(shape, 8, 10, "verify_i", [8192, 3001, 16, 5000], [7, 7, 3, 6], [6, 6, 2, 6], 7, seed_offset=4500)
+
+
 def test_llama2_13b_shape_two_layers():
     """Llama-2-13B layer shape (MHA, d 5120, ffn 13824, vocab 32000): two layers of the intermediate range,
     batch 2, context 2048, k = 6."""
