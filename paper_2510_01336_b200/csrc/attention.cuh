@@ -188,13 +188,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(2 * TILE) : "memory");
                         int row = (int)((((long long)p.pool_layer * p.n_pages + page) * p.hkv + kvh) * 16);
                         uint32_t dk = sm0 + s * 2 * TILE, dv = dk + TILE;
-#pragma unroll
-                        for (int h = 0; h < HALVES; ++h) {
-                            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                                         ::"r"(dk + h * 2048), "l"(&tmK), "r"(h * 64), "r"(row), "r"(fb) : "memory");
-                            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                                         ::"r"(dv + h * 2048), "l"(&tmV), "r"(h * 64), "r"(row), "r"(fb) : "memory");
-                        }
+                        // one copy per tensor: the page maps carry the head dimension's 64-element halves as a third
+                        // dimension, so the box covers the whole K (or V) page of this KV head
+                        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                                     ::"r"(dk), "l"(&tmK), "r"(0), "r"(row), "r"(0), "r"(fb) : "memory");
+                        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                                     ::"r"(dv), "l"(&tmV), "r"(0), "r"(row), "r"(0), "r"(fb) : "memory");
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;

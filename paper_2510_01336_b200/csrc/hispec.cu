@@ -125,9 +125,9 @@ struct hispec_ctx_ext {
     bool profiling;
     std::vector<ProfEvent> *prof;       // recorded since the last read
     std::vector<ProfEvent> *prof_free;  // event pairs ready for reuse
-    // tmK / tmV: rows of head_dim elements, box 64 x 16; tmK3 / tmV3: the same pages with the head dimension seen as
-    // [head_dim / 64][64], box 64 x 16 x (head_dim / 64): a whole K (or V) page of one KV head in one TMA copy
-    struct PageMaps { const void *k, *v; long long n_pages; int pool_layers; CUtensorMap tmK, tmV, tmK3, tmV3; } page_maps[4];
+    // tmK / tmV: the page pools as rows of head_dim elements with the head dimension seen as [head_dim / 64][64];
+    // box 64 x 16 x (head_dim / 64): a whole K (or V) page of one KV head in one TMA copy
+    struct PageMaps { const void *k, *v; long long n_pages; int pool_layers; CUtensorMap tmK, tmV; } page_maps[4];
     int n_page_maps;
     ActMapCache act_cache[3][8];
     int act_cache_n[3];
@@ -549,8 +549,7 @@ const hispec_ctx_ext::PageMaps *page_maps(hispec_ctx *c, const hispec_kv &kv) {
     int slot = x->n_page_maps < 4 ? x->n_page_maps++ : 3;
     auto &m = x->page_maps[slot];
     uint64_t rows = (uint64_t)kv.n_pool_layers * kv.n_pages * c->d.n_kv_heads * c->d.page_size;
-    if (!encode_2d(&m.tmK, kv.k_pages, c->d.head_dim, rows, 16) || !encode_2d(&m.tmV, kv.v_pages, c->d.head_dim, rows, 16) ||
-        !encode_pages3(&m.tmK3, kv.k_pages, c->d.head_dim, rows) || !encode_pages3(&m.tmV3, kv.v_pages, c->d.head_dim, rows)) {
+    if (!encode_pages3(&m.tmK, kv.k_pages, c->d.head_dim, rows) || !encode_pages3(&m.tmV, kv.v_pages, c->d.head_dim, rows)) {
         x->n_page_maps = slot;
         return nullptr;
     }
@@ -838,8 +837,8 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     wbytes *= m.n_rep;
     ProfScope prof(c, st, 20, wbytes);
     cudaError_t le = (d.head_dim == 64)
-                         ? cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK3, pm->tmV3, m)
-                         : cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK3, pm->tmV3, m);
+                         ? cudaLaunchKernelEx(&cfg, hispec_stage_kernel<64>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m)
+                         : cudaLaunchKernelEx(&cfg, hispec_stage_kernel<128>, *tmd, *tmo, *tmf, pm->tmK, pm->tmV, m);
     if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorLaunchOutOfResources) {
         // the GPU cannot hold one CTA per SM at once (e.g. it is shared): use the kernel sequence from now on
         (void)cudaGetLastError();
