@@ -12,9 +12,9 @@ library's CUDA kernels, called through the C ABI.
           the device time of K steps, all inputs resident in HBM, no host round trip;
   e2e     the same metric through the public driver with host buffers: per step the
           host reads the step's result record (device -> pinned host) and the tokens
-          are assembled on the host; prompt ids are uploaded from pinned host memory
-          (inside the timed region the per-step input is the pending token, which the
-          device already holds, so h2d bytes per step are 0 after the prompt);
+          are assembled on the host, and the next step's input -- the pending token, 4
+          bytes -- is uploaded from pinned host memory; the prompt ids were uploaded the
+          same way before the timed region;
   roofline  projections (the dominant kernel): weight bytes streamed / summed event
           time of the bracketed launches, against the measured HBM copy bandwidth;
   cpu_baseline  the fp32 CPU oracle timed on one super-round of the same shape.
@@ -152,6 +152,7 @@ def run_ours(args, rank, world, local_rank):
             loop.enqueue_super_round()
             if host_roundtrip:
                 loop.collect()
+                loop.push_pending()
         e1.record(stream)
         barrier()
         wall = time.perf_counter() - wall0
@@ -203,7 +204,7 @@ def run_ours(args, rank, world, local_rank):
                    "step_hbm_gbs": step_bytes / 1e9 / (ms / args.steps * 1e-3), "device_status": status,
                    "setup_s": round(setup_s, 1)},
         "clocks": sampler.summary(),
-        "e2e": {"value": toks_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
+        "e2e": {"value": toks_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4,
                 "d2h_bytes_per_step": 4 * (2 + max_rows + ROUNDS), "ms_per_step": ms_e2e / args.steps,
                 "prompt_h2d_bytes": 4 * N_PROMPT},
         "gpu_launches": launches,

@@ -128,6 +128,17 @@ class HiSpecLoop:
             self.stats.inter_accepted += int(self.h_acc_i[:, b].sum())
         return new
 
+    def push_pending(self, stream=None):
+        """Host-driven serving loop: upload, from pinned host memory, the token the host read back last as the next
+        draft input (4 bytes per sequence).  The acceptance kernel has left the same value on the device, so results
+        do not change; a caller that edits the token on the host (a stop rule, a forced token) uses this hook.
+        Must follow collect()."""
+        if not bool((self.h_next >= 0).all()):
+            return
+        s = stream if stream is not None else torch.cuda.current_stream()
+        with torch.cuda.stream(s):
+            self.pending.copy_(self.h_next, non_blocking=True)
+
     def generate(self, n_gen: int) -> List[List[int]]:
         while min(len(t) for t in self.tokens) < n_gen:
             self.enqueue_super_round()

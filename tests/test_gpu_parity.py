@@ -320,7 +320,7 @@ def test_tiny_adaptive_parameters_loop_is_lossless():
 
 
 @pytest.mark.parametrize("flagname,B", [("tcgen05", 3), ("simt", 3), ("rowwarp-attn", 3), ("multi-kernel", 3),
-                                        ("tcgen05", 20), ("tcgen05", 30)])
+                                        ("tcgen05", 12), ("tcgen05", 16), ("tcgen05", 20), ("tcgen05", 30)])
 def test_batched_ragged_gqa_pages_permuted(flagname, B):
     """GQA 2:1, head_dim 128, odd sizes (d 320, ffn 400, vocab 1000): a batch of 3 sequences with different
     context lengths, ragged row counts and scattered pages against the oracle, one sequence at a time;
@@ -328,8 +328,9 @@ def test_batched_ragged_gqa_pages_permuted(flagname, B):
     b = _binding()
     shape = wl.MINI_GQA
     w, m, hs = oracle_for(shape, kv_round=True)
-    # B = 20 gives 160 padded rows (the kernel-sequence path pairs two weight tiles per activation tile), B = 30
-    # gives 240 (one MMA per plane, separate accumulators)
+    # B = 12 and 16 give 96 and 128 padded rows (kernel-sequence path, one weight tile per CTA, one MMA over both
+    # planes), B = 20 gives 160 (two weight tiles per activation tile), B = 30 gives 240 (one MMA per plane, separate
+    # accumulators)
     N_d, max_rows, page = 4, 8, 16
     ctx_lens = ([37, 5, 64, 16, 33] * 6)[:B]
     n_rows = ([5, 3, 4, 1, 5] * 6)[:B]
