@@ -599,7 +599,11 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
     // an activation tile (gemm_pair_kernel), one CTA per SM; the K range is split so that the grid still fills the
     // GPU once.  Up to 128 rows the one-tile kernel (one MMA over both planes, two CTAs per SM) measured 2 % faster;
     // above 160 rows three stages of the pair no longer fit and it measured 4 % slower.
-    const int pair_rows = T_pad < 256 ? T_pad : 256;
+    // rows one launch can take: 256 (with hi/lo planes beyond 128 rows: one MMA per plane); more rows are cut into equal
+    // chunks (288 rows: 2 x 144, each in the pair kernel's window, instead of 256 + 32 -- every chunk streams the weights)
+    const int n_chunks = ceil_div(T_pad, 256);
+    const int chunk = T_pad <= 256 ? 256 : round_up(ceil_div(T_pad, n_chunks), 16);
+    const int pair_rows = T_pad < chunk ? T_pad : chunk;
     const bool pair_mode = !simt && planes == 2 && T_pad > 128 &&
                            3 * (2 * kWTileBytes + round_up(pair_rows, 16) * planes * 128) + 1024 <= kGemmMaxDynSmem;
     int splits = head ? 1 : p.splits;
@@ -612,7 +616,6 @@ int run_gemm(hispec_ctx *c, cudaStream_t st, GemmKind kind, const void *W, const
         while (splits > 1 && (size_t)splits * split_stride > c->part_floats) --splits;
     }
     if (splits_used) *splits_used = splits;
-    const int chunk = 256;   // rows one launch can take (with hi/lo planes beyond 128 rows: one MMA per plane)
     for (int row0 = 0; row0 < T_pad; row0 += chunk) {
         int rows = T_pad - row0 < chunk ? T_pad - row0 : chunk;
         ProfScope prof(c, st, 10 + (int)kind, 2.0 * (double)p.N * (double)p.K);
