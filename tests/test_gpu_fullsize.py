@@ -129,3 +129,82 @@ def test_llama3_8b_shape_plain_bf16_activations():
     """The same benchmarked call with plain bf16 tensor-core inputs (no hi/lo split): still inside the tolerances."""
     from paper_2510_01336_b200 import binding
     _run_case(wl.L3_8B, 8, 16, "verify_i", [1024], [6], [5], 13, flags=binding.FLAG_PLAIN_ACT)
+
+
+def test_llama3_8b_shape_draft_steps_batch1():
+    """The benchmarked draft calls, batch 1, context 1024, layers [0,8) + exit head L_d.
+    (1) Six draft steps + the bonus row as ONE launch (hispec_draft_block): the oracle runs the steps free, one after
+    the other; every step is compared (token, buffered exit row, appended K/V) until the first step whose greedy
+    token differs, which must be one the oracle's own top-2 margin leaves open (< 0.1).
+    (2) The same steps as single hispec_draft calls from the same start, each fed the ORACLE's token, so that all of
+    them are compared whatever the margins are."""
+    from paper_2510_01336_b200 import binding
+    shape, n_steps, c, page, max_rows = wl.L3_8B, 6, 1024, 16, 13
+    layers = list(range(0, shape.L_d))
+    w_gpu = wl.make_weights(shape, layers=layers, device="cuda", with_emb=True)
+    m = OracleModel.from_weights(w_gpu.to("cpu"), kv_round_bf16=True)
+    hs = HiSpecOracle(m, shape.L_d, shape.L_i, shape.L_f)
+    k_all, v_all, _ = wl.make_random_state(shape, layers, [c], max_rows, seed_offset=4600)
+    max_pages = (c + max_rows + page - 1) // page + 1
+    ctx = binding.Context(shape, w_gpu, page_size=page, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    t0 = int(wl.make_tokens(shape, 1, seed_offset=4601)[0])
+
+    def fresh():
+        st = ctx.new_state(1, max_pages + 3, wl.make_block_table(shape, 1, max_pages, n_pages=max_pages + 3),
+                           first_layer=0, n_pool_layers=len(layers))
+        for i, l in enumerate(layers):
+            gh.load_dense_kv(st, 0, i, k_all[i, 0, :c], v_all[i, 0, :c], page)
+        st.len_draft.fill_(c); st.len_inter.fill_(c); st.len_target.fill_(c)
+        return st
+
+    # the oracle's free run
+    ost = hs.new_state(c + max_rows + 1, max_rows)
+    for i, l in enumerate(layers):
+        ost.cache.k[l, :c] = k_all[i, 0, :c].float().numpy()
+        ost.cache.v[l, :c] = v_all[i, 0, :c].float().numpy()
+    ost.len_d = ost.len_i = ost.len_f = c
+    inputs, ref_tok, ref_margin = [t0], [], []
+    for j in range(n_steps + 1):
+        out = hs.draft_step(ost, inputs[j])
+        ref_tok.append(out.argmax_ids[0])
+        ref_margin.append(float(out.top2[0][0] - out.top2[0][1]))
+        inputs.append(out.argmax_ids[0])
+
+    def check_step(st, j, tag):
+        ref_row = ost.h_d[j].astype(np.float64)
+        rel = float(np.linalg.norm(st.h_draft[0, j].cpu().numpy() - ref_row) / np.linalg.norm(ref_row))
+        assert rel <= 1e-2, f"{tag} step {j}: buffered exit row rel-L2 {rel:.2e}"
+        gh.compare_kv(st, 0, ost, page, [layers[0], layers[-1]], [c + j], tag=f"{tag} step {j}")
+        return rel
+
+    # (1) one launch, free running
+    st = fresh()
+    S = torch.full((1, n_steps), -1, dtype=torch.int32, device="cuda")
+    ctx.draft_block(st, torch.tensor([t0], dtype=torch.int32, device="cuda"), S, n_steps, bonus=True)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    assert int(st.len_draft[0]) == c + n_steps + 1 and int(st.len_inter[0]) == c
+    got, compared, worst = S[0].tolist(), 0, 0.0
+    for j in range(n_steps + 1):          # the last step (bonus row) leaves no token
+        worst = max(worst, check_step(st, j, "block"))
+        compared += 1
+        if j < n_steps and got[j] != ref_tok[j]:
+            assert ref_margin[j] < 0.1, f"block step {j}: token {got[j]} != {ref_tok[j]} with margin {ref_margin[j]:.3f}"
+            break
+    assert compared >= 1
+    # (2) single calls, inputs from the oracle
+    st = fresh()
+    exempt = 0
+    for j in range(n_steps + 1):
+        tin = torch.tensor([inputs[j]], dtype=torch.int32, device="cuda")
+        tout = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        ctx.draft(st, tin, tout)
+        torch.cuda.synchronize()
+        worst = max(worst, check_step(st, j, "single"))
+        if int(tout[0]) != ref_tok[j]:
+            assert ref_margin[j] < 0.1, f"single step {j}: token {int(tout[0])} != {ref_tok[j]} with margin {ref_margin[j]:.3f}"
+            exempt += 1
+    assert ctx.status() == 0 and int(st.len_draft[0]) == c + n_steps + 1
+    print(f"\n[{shape.name} draft [0,{shape.L_d}) x {n_steps}+1] block steps compared {compared}, single steps "
+          f"{n_steps + 1} (exempt tokens {exempt}), worst row rel-L2 {worst:.2e}")
+    ctx.close()
