@@ -92,6 +92,8 @@ struct AttnTcArgs {
 };
 
 constexpr int kAttnStages = 4;
+// stacked query rows (G x R_pad) one CTA takes: up to eight 16-row warp tiles share every K / V page the CTA stages
+constexpr int kAttnGroupRows = 128;
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -129,7 +131,7 @@ __device__ __forceinline__ bool a_wait(uint32_t bar, uint32_t parity, volatile i
 }
 
 template <int HD>
-__global__ void __launch_bounds__(160)
+__global__ void __launch_bounds__((kAttnGroupRows / 16 + 1) * 32)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, StageArgs a,
                     RowMeta rm, AttnTcArgs p, uint32_t *status) {
     constexpr int HALVES = HD / 64;             // 128-byte column blocks per key row
@@ -201,8 +203,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             }
         }
     } else {
-        // ---- consumers: warp w owns stacked rows mg*64 + w*16 .. +15
-        const int r_lo = mg * 64 + warp * 16 + (lane >> 2), r_hi = r_lo + 8;
+        // ---- consumers: warp w owns stacked rows mg * kAttnGroupRows + w*16 .. +15
+        const int r_lo = mg * kAttnGroupRows + warp * 16 + (lane >> 2), r_hi = r_lo + 8;
         const int j_lo = r_lo / p.G, g_lo = r_lo % p.G, j_hi = r_hi / p.G, g_hi = r_hi % p.G;
         const bool v_lo = r_lo < QR && j_lo < nr, v_hi = r_hi < QR && j_hi < nr;
         const int kmax_lo = v_lo ? p0 + j_lo : -1, kmax_hi = v_hi ? p0 + j_hi : -1;
