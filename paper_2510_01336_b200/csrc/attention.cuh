@@ -134,7 +134,6 @@ template <int HD>
 __global__ void __launch_bounds__((kAttnGroupRows / 16 + 1) * 32)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, StageArgs a,
                     RowMeta rm, AttnTcArgs p, uint32_t *status) {
-    constexpr int HALVES = HD / 64;             // 128-byte column blocks per key row
     constexpr int TILE = 16 * HD * 2;           // bytes of one K (or V) page of one KV head
     constexpr int KS = HD / 16;                 // k-steps of Q K^T
     constexpr int NT = HD / 8;                  // n-tiles of P V

@@ -700,7 +700,7 @@ struct AttnSmem {
 template <int HD>
 __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, const MegaArgs &m, MegaShared &sh,
                                const AttnSmem sm_attn, int pool_layer, uint32_t &pg_it, int warp, int lane) {
-    constexpr int HALVES = HD / 64, TILE = 16 * HD * 2, KS = HD / 16, NT = HD / 8;
+    constexpr int TILE = 16 * HD * 2, KS = HD / 16, NT = HD / 8;
     const StageArgs &a = m.a;
     volatile int *abort_flag = &sh.abort_flag;
     const int per_b = m.n_splits * m.hkv * m.n_mg;
