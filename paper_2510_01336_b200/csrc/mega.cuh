@@ -729,10 +729,9 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
                 if (my < n_pg) pgid = m.block_table[(size_t)b * a.max_pages + pg0 + my];
                 if (my < n_pg && (pgid < 0 || pgid >= m.n_pages)) { atomicOr(m.status, HISPEC_ST_BOUNDS); pgid = 0; }
                 const int cnt = min(32, n_pg - i0);
-                for (int u = 0; u < cnt; ++u) {
+                for (int u = (int)((pw - (pg_it + (uint32_t)i0)) & 1u); u < cnt; u += 2) {   // this producer's pages
                     const long long page = __shfl_sync(0xffffffffu, pgid, u);
                     const uint32_t it = pg_it + i0 + u;
-                    if ((it & 1u) != pw) continue;
                     const int s = it & (uint32_t)(m.attn_stages - 1);
                     const uint32_t ph = (it >> m.attn_log2) & 1u;
                     if (lane == 0 && a_wait(a_smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, m.status)) {
@@ -784,11 +783,10 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             bool ok = true;
             const bool active = cw < m.mt;   // warps without rows only keep the page ring moving
             MEGA_STAMP(21);
-            for (int i = 0; i < n_pg && ok; ++i) {
+            // pages go to the warp groups (1, 2 or 4 of them) in turn by their running number; the number of stages is a
+            // multiple of the number of groups, so a stage always belongs to the same group and only its warps touch it
+            for (int i = (int)(((uint32_t)grp - pg_it) & (uint32_t)(m.ngrp - 1)); i < n_pg && ok; i += m.ngrp) {
                 const uint32_t it = pg_it + i;
-                // pages go to the warp groups in turn by their running number; the number of stages is a multiple of
-                // the number of groups, so a stage always belongs to the same group and only its warps touch it
-                if ((int)(it % (uint32_t)m.ngrp) != grp) continue;
                 const int s = it & (uint32_t)(m.attn_stages - 1);
                 const uint32_t ph = (it >> m.attn_log2) & 1u;
                 ok = a_wait(a_smem_u32(&sh.a_full[s]), ph, abort_flag, m.status);
