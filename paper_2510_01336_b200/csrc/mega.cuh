@@ -722,22 +722,25 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             // one issuing thread needs ~0.4 us per page, which bounded the phase on long contexts.  (A producer warp
             // whose 16 lanes each feed one stage and poll side by side measured 1 to 2 % slower than this.)
             const uint32_t pw = warp == kWarpX ? 0u : 1u;
+            // first row of this KV head in page 0 of the layer's pool, and the rows from one page to the next (a TMA
+            // coordinate is 32 bits wide, so the product fits)
+            const int row0 = (int)(((long long)pool_layer * m.n_pages * m.hkv + kvh) * 16), page_rows = m.hkv * 16;
             MEGA_STAMP(10);
             for (int i0 = 0; i0 < n_pg; i0 += 32) {
                 const int my = i0 + lane;
-                long long pgid = 0;
+                int pgid = 0;
                 if (my < n_pg) pgid = m.block_table[(size_t)b * a.max_pages + pg0 + my];
                 if (my < n_pg && (pgid < 0 || pgid >= m.n_pages)) { atomicOr(m.status, HISPEC_ST_BOUNDS); pgid = 0; }
                 const int cnt = min(32, n_pg - i0);
                 for (int u = (int)((pw - (pg_it + (uint32_t)i0)) & 1u); u < cnt; u += 2) {   // this producer's pages
-                    const long long page = __shfl_sync(0xffffffffu, pgid, u);
+                    const int page = __shfl_sync(0xffffffffu, pgid, u);
                     const uint32_t it = pg_it + i0 + u;
                     const int s = it & (uint32_t)(m.attn_stages - 1);
                     const uint32_t ph = (it >> m.attn_log2) & 1u;
                     if (lane == 0 && a_wait(a_smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, m.status)) {
                         const uint32_t fb = a_smem_u32(&sh.a_full[s]);
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fb), "r"(2 * TILE) : "memory");
-                        const int row = (int)((((long long)pool_layer * m.n_pages + page) * m.hkv + kvh) * 16);
+                        const int row = row0 + page * page_rows;
                         const uint32_t dk = sm_attn.at(s), dv = dk + TILE;
                         // one copy per tensor: the box spans the head dimension's 64-element halves as its third dimension
                         tma_load_3d(dk, tmK, 0, row, 0, fb);
