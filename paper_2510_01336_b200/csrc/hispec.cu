@@ -723,6 +723,8 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     double w_layer = 0.0;
     for (int k = 0; k < G_HEAD; ++k) w_layer += 2.0 * (double)c->plan[k].N * c->plan[k].K;
     if (kv_cap > w_layer && !env_int("HISPEC_FORCE_MEGA", 0)) return 1;
+    // the kernel's index arithmetic takes quotients of positions and item numbers below 2^21 through the reciprocal unit
+    if ((long long)d.max_pages_per_seq * d.page_size >= (1ll << 21) || (long long)a.batch * d.n_kv_heads * 64 * 16 >= (1ll << 21)) return 1;
     MegaArgs m;
     memset(&m, 0, sizeof(m));
     m.a = a;

@@ -213,6 +213,12 @@ __host__ __device__ inline void mega_slots(int tile, int tiles, int kbt, int G, 
     n_slots = (int)(((u1 + 1u) * Ge + U - 1u) / U) - 1 - first_cta + 1;
 }
 
+// Quotient of two small non-negative integers (x < 2^21, d >= 1) through the reciprocal unit: the index arithmetic of a
+// work item sits in front of its loads, on the critical path of every latency-bound phase, and a 32-bit integer
+// division by a run-time value is a chain of ~30 dependent instructions.  (x + 0.5) / d is at least 0.5 / d away from
+// an integer, the approximate division is off by at most 2 ulp, so truncation gives the exact quotient.
+__device__ __forceinline__ int qdiv(int x, int d) { return __float2int_rz(__fdividef((float)x + 0.5f, (float)d)); }
+
 // ---- barriers --------------------------------------------------------------------------------
 __device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kMegaWorkers) : "memory"); }
 
@@ -369,7 +375,7 @@ __device__ void ew_rows_in(const MegaArgs &m, MegaShared &sh, const float *gain,
     const StageArgs &a = m.a;
     const int nch = (m.d + kEwChunk - 1) / kEwChunk;
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
-        const int t = item / nch, ch = item % nch, b = t / a.R_pad, j = t % a.R_pad;
+        const int t = qdiv(item, nch), ch = item - t * nch, b = qdiv(t, a.R_pad), j = t - b * a.R_pad;
         const int c = ch * kEwChunk + lane * 8;
         bool valid = j < sh.nr[b];
         float v[8];
@@ -419,7 +425,7 @@ __device__ void ew_rope_table(const MegaArgs &m, MegaShared &sh, int gw, int ngw
     const StageArgs &a = m.a;
     const int half = m.hd / 2;
     for (int idx = (ngw - 1 - gw) * 32 + lane; idx < m.T_pad * half; idx += ngw * 32) {
-        const int t = idx / half, i = idx - t * half, b = t / a.R_pad, j = t - b * a.R_pad;
+        const int t = qdiv(idx, half), i = idx - t * half, b = qdiv(t, a.R_pad), j = t - b * a.R_pad;
         double sn, cs;
         sincos((double)(sh.p0[b] + j) * m.inv_freq[i], &sn, &cs);
         m.rope[idx] = make_float2((float)cs, (float)sn);
@@ -436,7 +442,7 @@ __device__ void ew_resid(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, i
     const int nch = (m.d + kSsqChunk - 1) / kSsqChunk;
     const int hl = lane >> 4, li = lane & 15;
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
-        const int t = item / nch, ch = item % nch, b = t / a.R_pad, j = t % a.R_pad;
+        const int t = qdiv(item, nch), ch = item - t * nch, b = qdiv(t, a.R_pad), j = t - b * a.R_pad;
         const int c = ch * kSsqChunk + li * 8;
         const bool valid = j < sh.nr[b];
         float ss = 0.f;
@@ -516,7 +522,7 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
     const int hd = m.hd, half = hd / 2, heads = m.hq + 2 * m.hkv, nq = m.hq * hd;
     const size_t stride = (size_t)m.T_pad * g.N;
     for (int item = gw; item < m.T_pad * heads; item += ngw) {
-        const int t = item / heads, h = item % heads, b = t / a.R_pad, j = t % a.R_pad;
+        const int t = qdiv(item, heads), h = item - t * heads, b = qdiv(t, a.R_pad), j = t - b * a.R_pad;
         if (j >= sh.nr[b]) {
             if (h < m.hq)
                 for (int i = lane; i < hd; i += 32) m.q[(size_t)t * nq + h * hd + i] = 0.f;
@@ -524,7 +530,7 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
         }
         const float ssq = mega_ssq_fetch(m, t, lane);
         const int pos = sh.p0[b] + j;
-        const int lp = pos / a.page_size, slot = pos % a.page_size;
+        const int lp = qdiv(pos, a.page_size), slot = pos - lp * a.page_size;
         // only loaded here: the check of the page id (a branch with a side effect) comes after the slot loads, which
         // must not wait for this load's round trip
         const long long page = m.block_table[(size_t)b * a.max_pages + lp];
@@ -595,7 +601,7 @@ __device__ void ew_qkv(const MegaArgs &m, MegaShared &sh, const MegaGemm &g, int
 __device__ void ew_silu(const MegaArgs &m, const MegaShared &sh, const MegaGemm &g, int gw, int ngw, int lane) {
     const int nch = (m.ffn + kEwChunk - 1) / kEwChunk;
     for (int item = gw; item < m.T_pad * nch; item += ngw) {
-        const int t = item / nch, ch = item % nch;
+        const int t = qdiv(item, nch), ch = item - t * nch;
         const int c = ch * kEwChunk + lane * 8;
         const float ssq = mega_ssq_fetch(m, t, lane);
         float gt[8], up[8], v[8];
@@ -626,7 +632,7 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
     const int nq = m.hq * HD;
     MEGA_STAMP(30);
     for (int item = gw; item < m.T_pad * m.hq; item += ngw) {
-        const int t = item / m.hq, h = item % m.hq, b = t / a.R_pad, j = t % a.R_pad;
+        const int t = qdiv(item, m.hq), h = item - t * m.hq, b = qdiv(t, a.R_pad), j = t - b * a.R_pad;
         float acc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
@@ -707,12 +713,12 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
     const int n_items = per_b * a.batch;
     const int QR = m.G * a.R_pad;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const int b = item / per_b, rest = item % per_b;
-        const int y = rest / m.n_splits, split = rest % m.n_splits;
-        const int kvh = y / m.n_mg, mg = y % m.n_mg;
+        const int b = qdiv(item, per_b), rest = item - b * per_b;
+        const int y = qdiv(rest, m.n_splits), split = rest - y * m.n_splits;
+        const int kvh = qdiv(y, m.n_mg), mg = y - kvh * m.n_mg;
         const int nr = sh.nr[b], p0 = sh.p0[b];
         const int total_pages = (p0 + nr + 15) >> 4;
-        int chunk = (total_pages + m.n_splits - 1) / m.n_splits;
+        int chunk = qdiv(total_pages + m.n_splits - 1, m.n_splits);
         if (chunk < 1) chunk = 1;
         const int pg0 = split * chunk, pg1 = min(pg0 + chunk, total_pages);
         const int n_pg = (nr > 0 && pg1 > pg0) ? pg1 - pg0 : 0;
@@ -756,7 +762,7 @@ __device__ void mega_attention(const CUtensorMap *tmK, const CUtensorMap *tmV, c
             const int mtp = 4 / m.ngrp;
             const int cw = (warp - kWarpEpi0) % mtp, grp = (warp - kWarpEpi0) / mtp;
             const int r_lo = mg * 64 + cw * 16 + (lane >> 2), r_hi = r_lo + 8;
-            const int j_lo = r_lo / m.G, g_lo = r_lo % m.G, j_hi = r_hi / m.G, g_hi = r_hi % m.G;
+            const int j_lo = qdiv(r_lo, m.G), g_lo = r_lo - j_lo * m.G, j_hi = qdiv(r_hi, m.G), g_hi = r_hi - j_hi * m.G;
             const bool v_lo = cw < m.mt && r_lo < QR && j_lo < nr, v_hi = cw < m.mt && r_hi < QR && j_hi < nr;
             const int kmax_lo = v_lo ? p0 + j_lo : -1, kmax_hi = v_hi ? p0 + j_hi : -1;
             const int nq = m.hq * HD;
@@ -1164,7 +1170,7 @@ __device__ __noinline__ void mega_store_logits(const MegaArgs &m, MegaShared &sh
         const int t = c0 + i;
         if (t >= m.T_pad) break;
         const float inv = mega_inv_rms_warp(m, t, lane);
-        const int b = t / m.a.R_pad, j = t % m.a.R_pad;
+        const int b = qdiv(t, m.a.R_pad), j = t - b * m.a.R_pad;
         if (n < N && j < sh.nr[b]) m.logits[((size_t)b * m.a.max_rows + j) * N + n] = v[i] * inv;
     }
 }
