@@ -412,3 +412,63 @@ def test_errors_and_status_word():
     torch.cuda.synchronize()
     assert ctx.status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("flagname", ["tcgen05", "multi-kernel"])
+def test_sequence_with_zero_rows_sits_out_and_all_empty_call(flagname):
+    """n_rows[b] == 0 skips sequence b: its length counters and its K/V pages stay as they were while its neighbours
+    are verified as usual; a call in which every sequence has zero rows changes nothing at all."""
+    b = _binding()
+    shape = wl.MINI_GQA
+    w, m, hs = oracle_for(shape, kv_round=True)
+    B, N_d, max_rows, page, max_pages = 3, 4, 8, 16, 8
+    ctx_lens, buffered = [37, 21, 64], [5, 3, 4]
+    n_rows, n_draft = [5, 0, 4], [4, 0, 4]
+    ctx = b.Context(shape, w.to("cuda"), page_size=page, max_batch=B, max_rows_per_seq=max_rows,
+                    max_pages_per_seq=max_pages, flags=FLAG_SETS[flagname])
+    states, drafts = [], []
+    for s in range(B):
+        prompt = wl.make_tokens(shape, ctx_lens[s], seed_offset=200 + s).tolist()
+        ost = hs.new_state(ctx_lens[s] + 16, max_rows)
+        pending = hs.prefill(ost, prompt).argmax_ids[0]
+        ar = hs.ar_generate(prompt, 8)
+        S = [ar[1 + j] if j < 2 else (ar[1 + j] + 7) % shape.vocab for j in range(4)]
+        u = pending
+        for t in (S + [None])[: buffered[s]]:
+            hs.draft_step(ost, u)
+            u = t
+        drafts.append(S)
+        states.append(ost)
+    bt = wl.make_block_table(shape, B, max_pages, n_pages=B * max_pages + 7, seed_offset=3100)
+    st = ctx.new_state(B, B * max_pages + 7, bt)
+    for s in range(B):
+        gh.load_seq(st, s, states[s], page, range(shape.n_layers), max_rows)
+    res = ctx.new_result(B, logits=True, hidden=True)
+    dt = torch.zeros((B, N_d), dtype=torch.int32)
+    for s in range(B):
+        dt[s, : len(drafts[s])] = torch.tensor(drafts[s], dtype=torch.int32)
+    i32 = lambda v: torch.tensor(v, dtype=torch.int32, device="cuda")
+    # every sequence empty: nothing moves
+    before = (st.len_draft.clone(), st.len_inter.clone(), st.len_target.clone(), st.k_pages.clone(), st.v_pages.clone())
+    ctx.verify_intermediate(st, dt.cuda(), i32([0, 0, 0]), i32([0, 0, 0]), res)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    for x, y in zip(before, (st.len_draft, st.len_inter, st.len_target, st.k_pages, st.v_pages)):
+        assert torch.equal(x, y)
+    # the middle sequence sits out
+    pages1 = st.block_table[1].long()
+    k1, v1 = st.k_pages[:, pages1].clone(), st.v_pages[:, pages1].clone()
+    ctx.verify_intermediate(st, dt.cuda(), i32(n_draft), i32(n_rows), res)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    import copy
+    for s in (0, 2):
+        ost = copy.deepcopy(states[s])
+        p0 = ost.len_i
+        out = hs.verify_intermediate(ost, drafts[s][: n_draft[s]], n_rows[s])
+        gh.compare_exit(out, res, s, n_rows[s], drafts[s][: n_draft[s]], check_accept=True, tag=f"seq{s}")
+        gh.compare_kv(st, s, ost, page, range(hs.L_d, hs.L_i), range(p0, p0 + n_rows[s]), tag=f"seq{s}")
+        assert int(st.len_inter[s]) == ost.len_i == int(st.len_draft[s])
+    assert int(st.len_draft[1]) == states[1].len_d and int(st.len_inter[1]) == states[1].len_i
+    assert torch.equal(st.k_pages[:, pages1], k1) and torch.equal(st.v_pages[:, pages1], v1)
+    ctx.close()
