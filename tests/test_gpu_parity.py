@@ -320,7 +320,7 @@ def test_tiny_adaptive_parameters_loop_is_lossless():
 
 
 @pytest.mark.parametrize("flagname,B", [("tcgen05", 3), ("simt", 3), ("rowwarp-attn", 3), ("multi-kernel", 3),
-                                        ("tcgen05", 12), ("tcgen05", 16), ("tcgen05", 20), ("tcgen05", 30)])
+                                        ("tcgen05", 12), ("tcgen05", 16), ("tcgen05", 20), ("tcgen05", 30), ("tcgen05", 64)])
 def test_batched_ragged_gqa_pages_permuted(flagname, B):
     """GQA 2:1, head_dim 128, odd sizes (d 320, ffn 400, vocab 1000): a batch of 3 sequences with different
     context lengths, ragged row counts and scattered pages against the oracle, one sequence at a time;
@@ -330,11 +330,11 @@ def test_batched_ragged_gqa_pages_permuted(flagname, B):
     w, m, hs = oracle_for(shape, kv_round=True)
     # B = 12 and 16 give 96 and 128 padded rows (kernel-sequence path, one weight tile per CTA, one MMA over both
     # planes), B = 20 gives 160 (two weight tiles per activation tile), B = 30 gives 240 (one MMA per plane, separate
-    # accumulators)
+    # accumulators), B = 64 -- the largest batch of the persistent kernel's tables -- gives 512 (two row chunks of 256)
     N_d, max_rows, page = 4, 8, 16
-    ctx_lens = ([37, 5, 64, 16, 33] * 6)[:B]
-    n_rows = ([5, 3, 4, 1, 5] * 6)[:B]
-    n_draft = ([4, 3, 4, 1, 4] * 6)[:B]
+    ctx_lens = ([37, 5, 64, 16, 33] * 13)[:B]
+    n_rows = ([5, 3, 4, 1, 5] * 13)[:B]
+    n_draft = ([4, 3, 4, 1, 4] * 13)[:B]
     max_pages = 8
     ctx = b.Context(shape, w.to("cuda"), page_size=page, max_batch=B, max_rows_per_seq=max_rows,
                     max_pages_per_seq=max_pages, flags=FLAG_SETS[flagname])
