@@ -84,8 +84,7 @@ int env_int(const char *name, int dflt) {
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
 
-// key splits of the tiled attention kernel: about four CTAs per SM over (batch, KV head, row group)
-// Key splits of the stand-alone attention kernel: about four CTAs per SM over the whole grid.  (Filling the CTA slots
+// Key splits of the stand-alone attention kernel: about four CTAs per SM over (batch, KV head, row group).  (Filling the CTA slots
 // exactly once instead -- fewer, longer CTAs -- is 2 % faster with equal contexts and 6 % slower with the ragged
 // contexts of a serving batch, whose longest sequences then form the tail.)
 inline int attn_splits(int sm_count, int batch, int hkv, int G, int R_pad) {

@@ -472,3 +472,44 @@ def test_sequence_with_zero_rows_sits_out_and_all_empty_call(flagname):
     assert int(st.len_draft[1]) == states[1].len_d and int(st.len_inter[1]) == states[1].len_i
     assert torch.equal(st.k_pages[:, pages1], k1) and torch.equal(st.v_pages[:, pages1], v1)
     ctx.close()
+
+
+def test_largest_batch_of_the_persistent_kernel_draft_step(monkeypatch):
+    """64 sequences (the persistent kernel's table size) with ragged contexts, one draft step each through layers
+    [0, L_d) + exit head as ONE launch: token (margin rule), buffered exit row, appended K/V and length counters of
+    every sequence against the oracle.  (With this toy model's weights the KV cache outweighs a layer, which would
+    route the call to the kernel sequence: the switch that keeps it on the persistent kernel is set.)"""
+    monkeypatch.setenv("HISPEC_FORCE_MEGA", "1")
+    b = _binding()
+    shape = wl.TINY
+    w, m, hs = oracle_for(shape, kv_round=True)
+    B, max_rows, page, max_pages = 64, 2, 16, 4
+    ctx = b.Context(shape, w.to("cuda"), page_size=page, max_batch=B, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages)
+    st = ctx.new_state(B, B * max_pages + 5, wl.make_block_table(shape, B, max_pages, n_pages=B * max_pages + 5, seed_offset=3200))
+    states, pend = [], []
+    for s in range(B):
+        n = 3 + (7 * s) % 40
+        prompt = wl.make_tokens(shape, n, seed_offset=300 + s).tolist()
+        ost = hs.new_state(n + 8, max_rows)
+        pend.append(hs.prefill(ost, prompt).argmax_ids[0])
+        states.append(ost)
+        gh.load_seq(st, s, ost, page, range(shape.n_layers), max_rows)
+    n0 = ctx.launch_count()
+    tin = torch.tensor(pend, dtype=torch.int32, device="cuda")
+    tout = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    ctx.draft(st, tin, tout)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0 and ctx.launch_count() - n0 == 1
+    got = tout.cpu().tolist()
+    for s in range(B):
+        ost = states[s]
+        p0 = ost.len_d
+        out = hs.draft_step(ost, pend[s])
+        if float(out.top2[0, 0] - out.top2[0, 1]) >= gh.MARGIN:
+            assert got[s] == out.argmax_ids[0], f"seq{s}: token"
+        row = st.h_draft[s, 0].cpu().numpy()
+        ref = ost.h_d[p0 - ost.len_i].astype(np.float64)
+        assert np.linalg.norm(row - ref) <= gh.HIDDEN_REL_L2 * np.linalg.norm(ref), f"seq{s}: buffered exit row"
+        gh.compare_kv(st, s, ost, page, range(0, hs.L_d), [p0], tag=f"seq{s}")
+        assert (int(st.len_draft[s]), int(st.len_inter[s]), int(st.len_target[s])) == (ost.len_d, ost.len_i, ost.len_f)
+    ctx.close()
