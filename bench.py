@@ -41,7 +41,7 @@ N_PROMPT, N_D, ROUNDS = 1024, 5, 2
 # workload: layers [8,16) + head, 6 rows, context 1024, 4.576 GB algorithmic) from the ncu capture summarised
 # under profiles/.  The launches of a super-round differ in size (a block of 6 draft steps, a verify-I, a
 # verify-T); their traffic is that ratio times their algorithmic bytes (traffic is the weight stream, read once).
-ROOFLINE_TRAFFIC_BYTES_CAPTURED = 4.627e9
+ROOFLINE_TRAFFIC_BYTES_CAPTURED = 4.628e9
 ROOFLINE_TRAFFIC_RATIO = ROOFLINE_TRAFFIC_BYTES_CAPTURED / 4.576e9
 
 
@@ -210,7 +210,7 @@ def run_ours(args, rank, world, local_rank):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": ROOFLINE_TRAFFIC_RATIO * roof_bytes / max(g_n, 1),
-                     "traffic_note": "ncu DRAM read+write of a verify-I launch (4.627 GB for 4.576 GB algorithmic), "
+                     "traffic_note": "ncu DRAM read+write of a verify-I launch (4.628 GB for 4.576 GB algorithmic), "
                                      "scaled to the average launch by algorithmic bytes",
                      "kernel": "hispec_stage_kernel (one launch = one block of draft steps, one verify-I or one verify-T call)",
                      "launches": g_n, "avg_launch_us": 1e3 * g_ms / max(g_n, 1),
