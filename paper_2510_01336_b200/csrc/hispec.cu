@@ -723,7 +723,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     for (int k = 0; k < G_HEAD; ++k) w_layer += 2.0 * (double)c->plan[k].N * c->plan[k].K;
     if (kv_cap > w_layer && !env_int("HISPEC_FORCE_MEGA", 0)) return 1;
     // the kernel's index arithmetic takes quotients of positions and item numbers below 2^21 through the reciprocal unit
-    if ((long long)d.max_pages_per_seq * d.page_size >= (1ll << 21) || (long long)a.batch * d.n_kv_heads * 64 * 16 >= (1ll << 21)) return 1;
+    if ((long long)d.max_pages_per_seq * d.page_size >= (1ll << 21)) return 1;
     MegaArgs m;
     memset(&m, 0, sizeof(m));
     m.a = a;
@@ -797,6 +797,7 @@ int run_stage_mega(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
     }
     if (m.n_splits < 1) m.n_splits = 1;
     if (m.n_splits > 16) m.n_splits = 16;
+    if ((long long)a.batch * d.n_kv_heads * m.n_mg * m.n_splits >= (1ll << 21)) return 1;   // attention item numbers, same rule
     m.ngrp = m.mt == 1 ? 4 : (m.mt == 2 ? 2 : 1);
     if (m.n_splits * m.ngrp > 32) m.ngrp = 32 / m.n_splits;   // one load batch in the split merge (16 splits: ngrp <= 2)
     if (m.ngrp == 3) m.ngrp = 2;
