@@ -551,7 +551,9 @@ const hispec_ctx_ext::PageMaps *page_maps(hispec_ctx *c, const hispec_kv &kv) {
     int slot = x->n_page_maps < 4 ? x->n_page_maps++ : 3;
     auto &m = x->page_maps[slot];
     uint64_t rows = (uint64_t)kv.n_pool_layers * kv.n_pages * c->d.n_kv_heads * c->d.page_size;
-    if (!encode_pages3(&m.tmK, kv.k_pages, c->d.head_dim, rows) || !encode_pages3(&m.tmV, kv.v_pages, c->d.head_dim, rows)) {
+    // (the kernels address a page row through a 32-bit TMA coordinate)
+    if (rows > 0x7fffffffull || !encode_pages3(&m.tmK, kv.k_pages, c->d.head_dim, rows) ||
+        !encode_pages3(&m.tmV, kv.v_pages, c->d.head_dim, rows)) {
         x->n_page_maps = slot;
         return nullptr;
     }
