@@ -894,7 +894,9 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         const GemmPlan &pq = c->plan[G_QKV], &po = c->plan[G_O], &pg = c->plan[G_GU], &pd = c->plan[G_DOWN];
         int sq = pq.splits, so = po.splits, sg = pg.splits, sd = pd.splits;
         if ((rc = run_gemm(c, st, G_QKV, c->wqkv[l], &c->tm_wqkv[l], 0, T_pad, sc, &sq)) != 0) return rc;
-        CK(launch(c, st, qkv_rope_store_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, sq,
+        // a thread per rotary pair: four times the threads where a row has the pairs to fill them
+        const int qk_threads = (d.n_q_heads + d.n_kv_heads) * (d.head_dim / 2) >= 1024 ? 1024 : 256;
+        CK(launch(c, st, qkv_rope_store_kernel, dim3(T_pad), dim3(qk_threads), 0, a, c->rows, (const float *)c->part, sq,
                   (size_t)T_pad * pq.N, d.n_q_heads, d.n_kv_heads, d.head_dim, (const double *)c->inv_freq, c->q,
                   (__nv_bfloat16 *)kv.k_pages, (__nv_bfloat16 *)kv.v_pages, kv.block_table, (long long)kv.n_pages,
                   pool_layer, c->status));
@@ -937,8 +939,10 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
                           (const float *)c->attn_part, ta.n_splits, d.n_q_heads, c->act_o, x->T_alloc, plain));
             }
         }
+        // one thread per four columns of the row, up to 1024 threads
+        const int rn_threads = d.d_model / 4 >= 1024 ? 1024 : (d.d_model / 4 <= 64 ? 64 : round_up(d.d_model / 4, 32));
         if ((rc = run_gemm(c, st, G_O, c->wo[l], &c->tm_wo[l], 1, T_pad, sc, &so)) != 0) return rc;
-        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, so,
+        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(rn_threads), 0, a, c->rows, (const float *)c->part, so,
                   (size_t)T_pad * po.N, c->ffn_norm[l], d.rms_eps, d.d_model, c->x, c->act_d, x->T_alloc, plain,
                   (float *)nullptr, (float *)nullptr));
         if ((rc = run_gemm(c, st, G_GU, c->wgu[l], &c->tm_wgu[l], 0, T_pad, sc, &sg)) != 0) return rc;
@@ -947,7 +951,7 @@ int run_stage(hispec_ctx *c, cudaStream_t st, const StageCall &sc) {
         if ((rc = run_gemm(c, st, G_DOWN, c->wdown[l], &c->tm_wdown[l], 2, T_pad, sc, &sd)) != 0) return rc;
         const bool last = (l + 1 == a.l1);
         const float *gain = last ? c->final_norm : c->attn_norm[l + 1];
-        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(256), 0, a, c->rows, (const float *)c->part, sd,
+        CK(launch(c, st, resid_norm_kernel, dim3(T_pad), dim3(rn_threads), 0, a, c->rows, (const float *)c->part, sd,
                   (size_t)T_pad * pd.N, gain, d.rms_eps, d.d_model, c->x, c->act_d, x->T_alloc, plain,
                   last ? exit_buf : (float *)nullptr, last ? hidden_out : (float *)nullptr));
     }
