@@ -139,10 +139,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     constexpr int NT = HD / 8;                  // n-tiles of P V
     __shared__ __align__(1024) uint8_t sm[kAttnStages * 2 * TILE];
     __shared__ __align__(8) uint64_t bar_full[kAttnStages], bar_empty[kAttnStages];
-    __shared__ int s_abort;
+    __shared__ int s_abort, s_seq;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int split = blockIdx.x, kvh = blockIdx.y / p.n_mg, mg = blockIdx.y % p.n_mg, b = blockIdx.z;
+    const int split = blockIdx.x, kvh = blockIdx.y / p.n_mg, mg = blockIdx.y % p.n_mg;
     volatile int *abort_flag = &s_abort;
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -156,6 +156,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     pdl_launch_dependents();
     pdl_wait();
 
+    // blockIdx.z counts the sequences from the longest to the shortest: blocks are dispatched in index order, so the
+    // long sequences of a ragged batch start first and the short ones fill the tail
+    for (int i = threadIdx.x; i < a.batch; i += blockDim.x) {
+        const int li = rm.p0[i] + rm.n_rows[i];
+        int rank = 0;
+        for (int j = 0; j < a.batch; ++j) {
+            const int lj = rm.p0[j] + rm.n_rows[j];
+            rank += (lj > li || (lj == li && j < i)) ? 1 : 0;
+        }
+        if (rank == (int)blockIdx.z) s_seq = i;
+    }
+    __syncthreads();
+    const int b = s_seq;
     const int nr = rm.n_rows[b], p0 = rm.p0[b];
     const int n_keys = p0 + nr;
     const int total_pages = (n_keys + 15) >> 4;
