@@ -643,6 +643,26 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
             float L = 0.f, M = -INFINITY;
             for (int s0 = 0; s0 < n_rec; s0 += 32) {
                 const int cnt = min(32, n_rec - s0);
+                // every load of the batch -- the lane's slice of up to 32 records and the (max, sum) pair of record
+                // s0 + lane -- is issued before the first use: one L2 round trip per batch (in groups of eight the
+                // loads of a group waited for the arithmetic of the one before: four round trips)
+                const float *r = base + (size_t)s0 * REC + lane * E;
+                float rv[32][E];
+#pragma unroll
+                for (int u = 0; u < 32; ++u) {
+                    if (u < cnt) {
+                        if constexpr (E == 4) {
+                            const float4 q4 = *reinterpret_cast<const float4 *>(r + (size_t)u * REC);
+                            rv[u][0] = q4.x; rv[u][1] = q4.y; rv[u][2] = q4.z; rv[u][3] = q4.w;
+                        } else {
+                            const float2 q2 = *reinterpret_cast<const float2 *>(r + (size_t)u * REC);
+                            rv[u][0] = q2.x; rv[u][1] = q2.y;
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) rv[u][e] = 0.f;
+                    }
+                }
                 float ms = -INFINITY, ls = 0.f;   // lane u holds (max, sum) of split s0 + u
                 if (lane < cnt) {
                     const float2 ml = *reinterpret_cast<const float2 *>(base + (size_t)(s0 + lane) * REC + HD);
@@ -658,22 +678,15 @@ __device__ void ew_attn_merge(const MegaArgs &m, MegaShared &sh, int gw, int ngw
 #pragma unroll
                 for (int e = 0; e < E; ++e) acc[e] *= corr;
                 const float wl = (ms == -INFINITY) ? 0.f : exp2f(ms - Mn);
-                const float *r = base + (size_t)s0 * REC + lane * E;
-#pragma unroll 8
-                for (int u = 0; u < cnt; ++u) {
-                    float rv[E];
-                    if constexpr (E == 4) {
-                        const float4 q4 = *reinterpret_cast<const float4 *>(r + (size_t)u * REC);
-                        rv[0] = q4.x; rv[1] = q4.y; rv[2] = q4.z; rv[3] = q4.w;
-                    } else {
-                        const float2 q2 = *reinterpret_cast<const float2 *>(r + (size_t)u * REC);
-                        rv[0] = q2.x; rv[1] = q2.y;
-                    }
-                    const float w = __shfl_sync(0xffffffffu, wl, u);
-                    const float l = __shfl_sync(0xffffffffu, ls, u);
-                    L += l * w;
 #pragma unroll
-                    for (int e = 0; e < E; ++e) acc[e] += w * rv[e];
+                for (int u = 0; u < 32; ++u) {
+                    if (u < cnt) {   // (warp-uniform)
+                        const float w = __shfl_sync(0xffffffffu, wl, u);
+                        const float l = __shfl_sync(0xffffffffu, ls, u);
+                        L += l * w;
+#pragma unroll
+                        for (int e = 0; e < E; ++e) acc[e] += w * rv[u][e];
+                    }
                 }
                 M = Mn;
             }
