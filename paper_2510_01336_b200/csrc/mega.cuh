@@ -990,6 +990,13 @@ struct WLane {
         cur_gi = ld.gi;
     }
 };
+// tensor map of projection number gi of the call (4 per layer, then the exit head; past the end: the first again,
+// which a block of draft steps comes back to) into the descriptor cache
+__device__ __forceinline__ void mega_prefetch_map(const MegaArgs &m, int gi, int n_g) {
+    if (gi >= n_g) gi = 0;
+    const MegaGemm *g = gi + 1 < n_g ? &m.gemms[(m.a.l0 + (gi >> 2)) * 4 + (gi & 3)] : m.head;
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&g->tmW) : "memory");
+}
 // attention phases that precede the projection the cursor stands in (only where the pages take the rings whole;
 // a pipeline without blocks in some projection skips it, so every projection computes its own count)
 __device__ __forceinline__ int mega_w_hold(const MegaArgs &m, const WCursor &c) {
@@ -1023,12 +1030,17 @@ __device__ __forceinline__ bool mega_w_issue(const MegaArgs &m, int p, WLane &w,
         w.cur_gi = w.ld.gi + w.ld.rep * w.ld.n_g;
         w.gate = true;
         w.hold = mega_w_hold(m, w.ld);
+        // the tensor map of the projection AFTER the one that starts now: a map's first use otherwise waits for its
+        // 128 bytes to come from memory, at the head of a phase
+        if (p == 0) mega_prefetch_map(m, w.ld.gi + 1, w.ld.n_g);
     }
     return true;
 }
 __device__ __forceinline__ void mega_w_producer(const MegaArgs &m, const MegaRing *ring, MegaShared &sh) {
     volatile int *ab = &sh.abort_flag;
     WLane w0(&m, &sh, 0), w1(&m, &sh, 1);
+    mega_prefetch_map(m, 0, w0.ld.n_g);
+    mega_prefetch_map(m, 1, w0.ld.n_g);
     w0.hold = mega_w_hold(m, w0.ld);
     w1.hold = mega_w_hold(m, w1.ld);
     // weights are read exactly once per call: mark their lines evict-first so that they do not push the
