@@ -220,3 +220,34 @@ def test_llama3_8b_shape_draft_steps_batch1():
     print(f"\n[{shape.name} draft [0,{shape.L_d}) x {n_steps}+1] block steps compared {compared}, single steps "
           f"{n_steps + 1} (exempt tokens {exempt}), worst row rel-L2 {worst:.2e}")
     ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_small_calls_against_the_oracle(seed, monkeypatch):
+    """Seeded random calls on the two toy shapes (head_dim 64 MHA and head_dim 128 GQA): random batch size, ragged row
+    counts, contexts that include zero, one and page-boundary lengths, either verification call, either GPU path --
+    each compared with the oracle exactly as the full-size cases are."""
+    import dataclasses
+    from paper_2510_01336_b200 import binding
+    monkeypatch.setenv("HISPEC_FORCE_MEGA", "1")   # toy weights: keep KV-heavy calls on the persistent kernel
+    rng = np.random.default_rng(2000 + seed)
+    shape = (wl.TINY, wl.MINI_GQA)[seed % 2]
+    kind = ("verify_i", "verify_t")[(seed // 2) % 2]
+    flags = (0, binding.FLAG_MULTI_KERNEL)[(seed // 4) % 2]
+    max_rows = 8
+    B = int(rng.integers(1, 7))
+    special = [0, 1, 15, 16, 17, 32, 47, 48, 49, 100]
+    ctx_lens = [int(rng.choice(special)) if rng.random() < 0.6 else int(rng.integers(0, 110)) for _ in range(B)]
+    if max(ctx_lens) == 0:
+        ctx_lens[0] = 33
+    if kind == "verify_i":
+        n_draft = [int(rng.integers(0, max_rows)) for _ in range(B)]
+        n_rows = [d + int(rng.integers(0, 2)) if d else 1 for d in n_draft]      # with or without the bonus row
+        n_rows = [min(r, max_rows) for r in n_rows]
+        n_draft = [min(d, r) for d, r in zip(n_draft, n_rows)]
+        l0, l1 = shape.L_d, shape.L_i
+    else:
+        n_rows = [int(rng.integers(1, max_rows)) for _ in range(B)]
+        n_draft = list(n_rows)
+        l0, l1 = shape.L_i, shape.L_f
+    _run_case(shape, l0, l1, kind, ctx_lens, n_rows, n_draft, max_rows, flags=flags, seed_offset=8000 + 10 * seed)
