@@ -18,6 +18,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--calls", type=int, default=3)
     ap.add_argument("--rows", type=int, default=6)
+    ap.add_argument("--batch", type=int, default=1, help="sequences in the call (rows and context apply to each)")
     ap.add_argument("--ctx", type=int, default=1024)
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--shape", default="llama3-8b-shape", choices=sorted(wl.SHAPES),
@@ -26,20 +27,21 @@ def main():
     shape = wl.SHAPES[args.shape]
     layers = list(range(shape.L_d, shape.L_i))
     w = wl.make_weights(shape, layers=layers, device="cuda", with_emb=False)
-    max_rows = 13
+    B = args.batch
+    max_rows = 13 if B == 1 else args.rows
     max_pages = (args.ctx + max_rows + 15) // 16 + 1
-    ctx = binding.Context(shape, w, page_size=16, max_batch=1, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages,
+    ctx = binding.Context(shape, w, page_size=16, max_batch=B, max_rows_per_seq=max_rows, max_pages_per_seq=max_pages,
                           flags=args.flags)
-    st = ctx.new_state(1, max_pages, wl.make_block_table(shape, 1, max_pages), first_layer=shape.L_d,
+    st = ctx.new_state(B, B * max_pages, wl.make_block_table(shape, B, max_pages), first_layer=shape.L_d,
                        n_pool_layers=len(layers))
     g = torch.Generator(device="cuda").manual_seed(shape.seed + 4000)
     st.k_pages.normal_(generator=g)
     st.v_pages.normal_(generator=g)
     st.h_draft.normal_(generator=g)
-    res = ctx.new_result(1)
+    res = ctx.new_result(B)
     i32 = lambda v: torch.tensor(v, dtype=torch.int32, device="cuda")
-    drafts = torch.zeros((1, max_rows - 1), dtype=torch.int32, device="cuda")
-    nd, nr = i32([args.rows - 1]), i32([args.rows])
+    drafts = torch.zeros((B, max(max_rows - 1, 1)), dtype=torch.int32, device="cuda")
+    nd, nr = i32([args.rows - 1] * B), i32([args.rows] * B)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.calls + 1)]
     ev[0].record()
     for i in range(args.calls):
@@ -50,10 +52,10 @@ def main():
         ev[i + 1].record()
     torch.cuda.synchronize()
     status = ctx.status()
-    by = len(layers) * shape.layer_weight_bytes + shape.head_bytes + len(layers) * shape.kv_bytes_per_token_layer * (args.ctx + args.rows)
+    by = len(layers) * shape.layer_weight_bytes + shape.head_bytes + B * len(layers) * shape.kv_bytes_per_token_layer * (args.ctx + args.rows)
     for i in range(args.calls):
         ms = ev[i].elapsed_time(ev[i + 1])
-        print(f"{shape.name} [{shape.L_d},{shape.L_i}) rows {args.rows} ctx {args.ctx} call {i}: {ms * 1e3:.1f} us, "
+        print(f"{shape.name} [{shape.L_d},{shape.L_i}) batch {B} rows {args.rows} ctx {args.ctx} call {i}: {ms * 1e3:.1f} us, "
               f"{by / 1e9:.2f} GB, {by / ms / 1e6:.0f} GB/s algorithmic, status {status}")
     ctx.close()
 
